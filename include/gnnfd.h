@@ -1,0 +1,183 @@
+/*
+ * gnnfd — feature-decomposed GNN aggregation on one CUDA device (sm_100a).
+ *
+ * The library computes the Aggregation phase of message-passing GNN inference
+ * (Algorithm 1, the loop over decomposition layers p with its Message,
+ * Aggregate and Concat steps): the feature dimension is cut into chunks of
+ * `chunk_width` columns, every chunk is aggregated over all vertices, and each
+ * chunk's result is written into its own columns of the output.  The
+ * Combination (dense) phase is the caller's; its output is this library's input
+ * (Section III: combination is run ahead of aggregation).
+ *
+ * Conventions
+ *   - Every pointer named d_* is DEVICE memory owned by the caller.  The library
+ *     never allocates or frees device memory; it carves what it needs out of
+ *     the buffers it is handed.  Host pointers are named without the prefix.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - All entry points return a gnnfd_status_t (0 = success, negative = error);
+ *     nothing throws, aborts or traps.  Device-side problems (a vertex id out of
+ *     range) are counted on the device and reported as a status.
+ *   - Matrices are row-major with a leading dimension in ELEMENTS (ld >= width).
+ *     Padding columns are never written and never influence a result.
+ *   - Same inputs give bit-identical outputs from run to run: no floating-point
+ *     atomics are used anywhere.
+ *   - Graph structure is int32 on the device: n and nnz must stay below 2^31.
+ */
+#ifndef GNNFD_H
+#define GNNFD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gnnfd_csr gnnfd_csr_t; /* opaque host-side handle; holds device pointers into caller memory */
+
+typedef enum { GNNFD_F32 = 0, GNNFD_BF16 = 1 } gnnfd_dtype_t;
+typedef enum { GNNFD_I32 = 0, GNNFD_I64 = 1 } gnnfd_itype_t;
+
+/* gnnfd_build_csr flags */
+enum {
+    GNNFD_CSR_ADD_SELF_LOOPS = 1, /* drop every input loop, then add exactly one (v,v) per vertex */
+    GNNFD_CSR_DEDUP = 2,          /* keep the first (lowest edge id) of equal (dst, src) pairs */
+    GNNFD_CSR_SYMMETRIZE = 4      /* add the reverse of every non-loop edge, with edge id e + i */
+};
+
+typedef enum {
+    GNNFD_OK = 0,
+    GNNFD_INVALID_ARG = -1,         /* null pointer, non-positive size, ld < width, heads*dim mismatch */
+    GNNFD_BAD_INDEX = -2,           /* a vertex id outside [0, n) was found in the edge list */
+    GNNFD_TOO_LARGE = -3,           /* n, e or the resulting nnz does not fit the int32 structure */
+    GNNFD_WORKSPACE_TOO_SMALL = -4, /* a caller-provided buffer is smaller than the size query says */
+    GNNFD_UNSUPPORTED = -5,         /* unknown dtype / itype enum */
+    GNNFD_CUDA_ERROR = -6           /* a CUDA runtime call failed; see gnnfd_last_cuda_error() */
+} gnnfd_status_t;
+
+/* ------------------------------------------------------------------ graph set-up
+ *
+ * CSR by destination from a COO edge list (Section II-C: the aggregation's input
+ * is the edge set in COO form plus the vertex features).  Edge i goes from
+ * src[i] to dst[i]; row v of the CSR lists the sources of the edges that end in
+ * v.  Steps, in this order: reject ids outside [0,n); SYMMETRIZE; ADD_SELF_LOOPS;
+ * order by (dst, src), ties by ascending edge id; DEDUP.  Besides row_ptr /
+ * col_idx the build stores perm (CSR slot -> input edge id; e + i for the
+ * reverse of edge i; -1 for an added self-loop), the degree normalisers
+ * deg^-1/2 and 1/deg (0 for empty rows, deg = entries in the row), the GCN edge
+ * weight deg(src)^-1/2 * deg(dst)^-1/2 per slot, and the launch schedule (rows
+ * grouped by degree, rows above GNNFD_HUB_DEGREE cut into segments of
+ * GNNFD_HUB_SEGMENT edges).
+ */
+#define GNNFD_HUB_DEGREE 2048
+#define GNNFD_HUB_SEGMENT 1024
+
+/* Sizes (bytes) of the two device buffers gnnfd_build_csr needs for n vertices and e input edges.
+ * persistent: must stay alive and untouched while the handle is in use.
+ * scratch:    only during the call. */
+int gnnfd_csr_workspace_bytes(int64_t n, int64_t e, uint32_t flags, size_t* persistent_bytes,
+                              size_t* scratch_bytes);
+
+/* Builds the CSR.  d_src / d_dst: device arrays of e vertex ids of type `itype`, not modified.
+ * d_persistent / d_scratch: device buffers, 256-byte aligned, at least as large as the size query
+ * says.  Enqueues on `stream` and synchronises it once before returning (the host needs nnz and
+ * the bad-index count).  On success *out receives a new handle (release with gnnfd_csr_destroy;
+ * the device memory stays the caller's).  On GNNFD_BAD_INDEX no handle is produced. */
+int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, gnnfd_itype_t itype,
+                    uint32_t flags, void* d_persistent, size_t persistent_bytes, void* d_scratch,
+                    size_t scratch_bytes, void* stream, gnnfd_csr_t** out);
+
+/* Reads the handle.  Any output pointer may be NULL.  The d_* results point into d_persistent:
+ * row_ptr[n+1], col_idx[nnz], perm[nnz], dinv_sqrt[n], rdeg[n], edge_weight[nnz]. */
+int gnnfd_csr_info(const gnnfd_csr_t* csr, int64_t* n, int64_t* nnz, const int32_t** d_row_ptr,
+                   const int32_t** d_col_idx, const int32_t** d_perm, const float** d_dinv_sqrt,
+                   const float** d_rdeg, const float** d_edge_weight, int32_t* max_degree);
+
+/* The launch schedule.  bin_count[5]: rows with degree <= 8, <= 32, <= 128, <= GNNFD_HUB_DEGREE, and
+ * hub rows.  d_row_order[n]: row ids grouped by bin (ascending id inside a bin).  Hub segments:
+ * d_seg_row[n_segments], d_seg_begin[n_segments] (first CSR slot of the segment);
+ * d_hub_seg_ptr[n_hub+1] indexes the segments of the i-th hub row (i-th row of the last bin). */
+int gnnfd_csr_schedule(const gnnfd_csr_t* csr, int64_t bin_count[5], const int32_t** d_row_order,
+                       int64_t* n_segments, const int32_t** d_seg_row, const int32_t** d_seg_begin,
+                       const int32_t** d_hub_seg_ptr);
+
+/* Frees the host-side handle only. */
+void gnnfd_csr_destroy(gnnfd_csr_t* csr);
+
+/* ------------------------------------------------------------------ GCN / GraphSAGE aggregation
+ *
+ * out[v, j] = s_v * sum over the CSR entries k of row v of w_k * x[col_idx[k], j]
+ *   GCN : w_k = deg(col_idx[k])^-1/2 * deg(v)^-1/2, s_v = 1   (with the self-loop flag this is
+ *         the symmetric normalisation D^-1/2 (A + I) D^-1/2 X of the cited GCN model)
+ *   SAGE: w_k = 1, s_v = 1/deg(v)                              (neighbourhood mean)
+ * Empty rows give 0.  Products and sums are fp32 (bf16 inputs are widened exactly).
+ *
+ * chunk_width (>= 1) is the width of one decomposition layer: P = ceil(f / chunk_width) chunks, the
+ * last one narrower; chunk_width >= f means no decomposition.  Chunks are swept one after the other
+ * over all rows, so the gathered working set of a sweep is n * chunk_width elements.  The result
+ * does not depend on chunk_width beyond fp32 rounding of identical sums (it is in fact bit-identical).
+ *
+ * d_x: [n, ldx] of xdt.  d_out: [n, ldo] of odt (must not alias d_x).  d_scratch: per-call buffer
+ * of gnnfd_aggregate_workspace_bytes(csr, f) bytes (holds the per-segment partial sums of hub rows;
+ * 0 bytes when the graph has no hub row, NULL is then accepted).  The call only enqueues work.
+ * 16-byte-aligned pointers with ldx*sizeof(x) and chunk offsets multiples of 16 bytes take the
+ * 128-bit load path; anything else is still correct through narrower loads. */
+int gnnfd_aggregate_workspace_bytes(const gnnfd_csr_t* csr, int32_t f, size_t* scratch_bytes);
+
+int gnnfd_aggregate_gcn(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt,
+                        void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
+                        void* d_scratch, size_t scratch_bytes, void* stream);
+
+int gnnfd_aggregate_sage(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt,
+                         void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
+                         void* d_scratch, size_t scratch_bytes, void* stream);
+
+/* ------------------------------------------------------------------ GAT
+ *
+ * Scores (full head width, computed once, never per chunk):
+ *   s_src[u, h] = sum_d a_src[h, d] * z[u, h*dim + d],   s_dst[v, h] likewise with a_dst.
+ * Logit of CSR entry k of row v, head h: LeakyReLU(s_src[col_idx[k], h] + s_dst[v, h]) with the given
+ * negative slope.  alpha = softmax of the logits over the entries of the row (multi-edges are
+ * separate terms).  out[v, h*dim + d] = sum_k alpha[k, h] * z[col_idx[k], h*dim + d]; empty row -> 0.
+ * The fused kernel evaluates logits, a running (max, sum) softmax and the weighted sum in one pass
+ * over the row; chunk_width decomposes the flattened heads*dim columns (column j uses head j / dim).
+ */
+
+/* d_z [n, ldz] of zdt; d_a_src / d_a_dst [heads, dim] fp32; d_s_src / d_s_dst [n, heads] fp32 out. */
+int gnnfd_gat_scores(int64_t n, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
+                     const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst,
+                     void* stream);
+
+/* Scratch for gnnfd_aggregate_gat: the two score arrays plus hub-row partials. */
+int gnnfd_gat_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, size_t* scratch_bytes);
+
+int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt,
+                        const float* d_a_src, const float* d_a_dst, int32_t heads, int32_t dim,
+                        float negative_slope, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                        int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
+
+/* alpha[k, h] for every CSR slot k, [nnz, heads] fp32 in CSR order, from caller-supplied scores. */
+int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
+                       float negative_slope, float* d_alpha, void* stream);
+
+/* ------------------------------------------------------------------ diagnostics */
+
+const char* gnnfd_status_string(int status);
+
+/* cudaError_t of the most recent failed runtime call made by this library on this thread (0 if none). */
+int gnnfd_last_cuda_error(void);
+
+/* Kernels launched by this library since it was loaded. */
+int64_t gnnfd_launch_count(void);
+
+/* Optional per-kernel timing.  While enabled every launch is bracketed by CUDA events on its stream.
+ * gnnfd_kernel_timing_read synchronises the recorded events, clears them, and fills up to `capacity`
+ * entries: names[i] (static strings), ms[i] (total milliseconds), launches[i].  Returns the number of
+ * distinct kernels seen (may exceed capacity), or a negative status. */
+int gnnfd_kernel_timing_enable(int on);
+int gnnfd_kernel_timing_read(const char** names, double* ms, int64_t* launches, int capacity);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GNNFD_H */

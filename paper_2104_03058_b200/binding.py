@@ -1,0 +1,295 @@
+"""Thin ctypes binding of libgnnfd.so: argument marshalling only.
+
+PyTorch supplies device memory and streams; every step of the aggregation runs inside the library's
+CUDA kernels.  There is no fallback: if the shared library is missing or fails to load, importing
+the entry points raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+I32, I64 = 0, 1
+CSR_ADD_SELF_LOOPS, CSR_DEDUP, CSR_SYMMETRIZE = 1, 2, 4
+OK, INVALID_ARG, BAD_INDEX, TOO_LARGE, WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA_ERROR = 0, -1, -2, -3, -4, -5, -6
+HUB_DEGREE, HUB_SEGMENT = 2048, 1024
+
+_lib = None
+
+
+class GnnfdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().gnnfd_status_string(status).decode()
+        if status == CUDA_ERROR:
+            msg += " (cudaError %d)" % lib().gnnfd_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg))
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgnnfd.so from the package directory (never builds, never falls back)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise ImportError("libgnnfd.so is not built: run paper_2104_03058_b200.build.build_library()")
+        L = ctypes.CDLL(path)
+        i64, i32, u32, vp, sz, fl = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32, ctypes.c_void_p,
+                                     ctypes.c_size_t, ctypes.c_float)
+        pp = ctypes.POINTER
+        L.gnnfd_csr_workspace_bytes.argtypes = [i64, i64, u32, pp(sz), pp(sz)]
+        L.gnnfd_build_csr.argtypes = [i64, i64, vp, vp, i32, u32, vp, sz, vp, sz, vp, pp(vp)]
+        L.gnnfd_csr_info.argtypes = [vp, pp(i64), pp(i64), pp(vp), pp(vp), pp(vp), pp(vp), pp(vp), pp(vp), pp(i32)]
+        L.gnnfd_csr_schedule.argtypes = [vp, pp(i64 * 5), pp(vp), pp(i64), pp(vp), pp(vp), pp(vp)]
+        L.gnnfd_csr_destroy.argtypes = [vp]
+        L.gnnfd_csr_destroy.restype = None
+        L.gnnfd_aggregate_workspace_bytes.argtypes = [vp, i32, pp(sz)]
+        agg = [vp, vp, i64, i32, vp, i64, i32, i32, i32, vp, sz, vp]
+        L.gnnfd_aggregate_gcn.argtypes = agg
+        L.gnnfd_aggregate_sage.argtypes = agg
+        L.gnnfd_gat_scores.argtypes = [i64, vp, i64, i32, vp, vp, i32, i32, vp, vp, vp]
+        L.gnnfd_gat_workspace_bytes.argtypes = [vp, i32, i32, pp(sz)]
+        L.gnnfd_aggregate_gat.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32, vp, sz, vp]
+        L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp]
+        L.gnnfd_status_string.argtypes = [ctypes.c_int]
+        L.gnnfd_status_string.restype = ctypes.c_char_p
+        L.gnnfd_last_cuda_error.restype = ctypes.c_int
+        L.gnnfd_launch_count.restype = i64
+        L.gnnfd_kernel_timing_enable.argtypes = [ctypes.c_int]
+        L.gnnfd_kernel_timing_read.argtypes = [pp(ctypes.c_char_p), pp(ctypes.c_double), pp(i64), ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise GnnfdError(status, where)
+
+
+def _stream_ptr(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("features must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _matrix(t: torch.Tensor, cols: int, name: str):
+    """(pointer, leading dimension) of a row-major device matrix with at least `cols` columns."""
+    if not t.is_cuda or t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1) or t.shape[1] < cols:
+        raise ValueError("%s must be a 2-D CUDA tensor with unit column stride and >= %d columns" % (name, cols))
+    return ctypes.c_void_p(t.data_ptr()), t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _alloc_bytes(nbytes: int, device) -> torch.Tensor:
+    # torch's caching allocator returns 512-byte aligned blocks
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+class Csr:
+    """Handle of a built CSR; keeps the persistent device buffer alive."""
+
+    def __init__(self, handle, persistent: torch.Tensor, device):
+        self._h = handle
+        self._persistent = persistent
+        self.device = device
+        n, nnz, md = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32()
+        ptrs = [ctypes.c_void_p() for _ in range(6)]
+        _check(lib().gnnfd_csr_info(self._h, ctypes.byref(n), ctypes.byref(nnz), *[ctypes.byref(p) for p in ptrs],
+                                    ctypes.byref(md)), "gnnfd_csr_info")
+        self.n, self.nnz, self.max_degree = n.value, nnz.value, md.value
+        self._ptrs = dict(zip(("row_ptr", "col_idx", "perm", "dinv_sqrt", "rdeg", "edge_weight"),
+                              [p.value for p in ptrs]))
+        bins = (ctypes.c_int64 * 5)()
+        nseg = ctypes.c_int64()
+        sp = [ctypes.c_void_p() for _ in range(4)]
+        _check(lib().gnnfd_csr_schedule(self._h, ctypes.byref(bins), ctypes.byref(sp[0]), ctypes.byref(nseg),
+                                        ctypes.byref(sp[1]), ctypes.byref(sp[2]), ctypes.byref(sp[3])),
+               "gnnfd_csr_schedule")
+        self.bin_count = list(bins)
+        self.n_segments = nseg.value
+        self._ptrs.update(dict(zip(("row_order", "seg_row", "seg_begin", "hub_seg_ptr"), [p.value for p in sp])))
+
+    @property
+    def handle(self):
+        if self._h is None:
+            raise RuntimeError("CSR handle was destroyed")
+        return self._h
+
+    def _view(self, name: str, count: int, dtype) -> torch.Tensor:
+        """A tensor view (no copy) of one of the arrays inside the persistent buffer."""
+        off = self._ptrs[name] - self._persistent.data_ptr()
+        size = torch.empty(0, dtype=dtype).element_size()
+        return self._persistent[off:off + count * size].view(dtype)
+
+    row_ptr = property(lambda self: self._view("row_ptr", self.n + 1, torch.int32))
+    col_idx = property(lambda self: self._view("col_idx", self.nnz, torch.int32))
+    perm = property(lambda self: self._view("perm", self.nnz, torch.int32))
+    dinv_sqrt = property(lambda self: self._view("dinv_sqrt", self.n, torch.float32))
+    rdeg = property(lambda self: self._view("rdeg", self.n, torch.float32))
+    edge_weight = property(lambda self: self._view("edge_weight", self.nnz, torch.float32))
+    row_order = property(lambda self: self._view("row_order", self.n, torch.int32))
+    seg_row = property(lambda self: self._view("seg_row", self.n_segments, torch.int32))
+    seg_begin = property(lambda self: self._view("seg_begin", self.n_segments, torch.int32))
+    hub_seg_ptr = property(lambda self: self._view("hub_seg_ptr", self.bin_count[4] + 1, torch.int32))
+
+    def destroy(self):
+        if self._h is not None:
+            lib().gnnfd_csr_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def csr_workspace_bytes(n: int, e: int, flags: int):
+    p, s = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().gnnfd_csr_workspace_bytes(n, e, flags, ctypes.byref(p), ctypes.byref(s)), "gnnfd_csr_workspace_bytes")
+    return p.value, s.value
+
+
+def build_csr(n: int, src: torch.Tensor, dst: torch.Tensor, flags: int = 0, stream=None,
+              persistent: torch.Tensor | None = None, scratch: torch.Tensor | None = None) -> Csr:
+    """gnnfd_build_csr on device tensors src/dst (int32 or int64, same dtype and length)."""
+    if not (src.is_cuda and dst.is_cuda) or src.dtype != dst.dtype or src.shape != dst.shape or src.dim() != 1:
+        raise ValueError("src and dst must be 1-D CUDA tensors of the same dtype and length")
+    if src.dtype not in (torch.int32, torch.int64):
+        raise TypeError("edge ids must be int32 or int64")
+    src, dst = src.contiguous(), dst.contiguous()
+    e = src.numel()
+    pb, sb = csr_workspace_bytes(n, e, flags)
+    if persistent is None:
+        persistent = _alloc_bytes(pb, src.device)
+    if scratch is None:
+        scratch = _alloc_bytes(sb, src.device)
+    handle = ctypes.c_void_p()
+    st = lib().gnnfd_build_csr(n, e, ctypes.c_void_p(src.data_ptr()), ctypes.c_void_p(dst.data_ptr()),
+                               I32 if src.dtype == torch.int32 else I64, flags,
+                               ctypes.c_void_p(persistent.data_ptr()), persistent.numel(),
+                               ctypes.c_void_p(scratch.data_ptr()), scratch.numel(), _stream_ptr(stream),
+                               ctypes.byref(handle))
+    _check(st, "gnnfd_build_csr")
+    return Csr(handle, persistent, src.device)
+
+
+def aggregate_workspace_bytes(csr: Csr, f: int) -> int:
+    s = ctypes.c_size_t()
+    _check(lib().gnnfd_aggregate_workspace_bytes(csr.handle, f, ctypes.byref(s)), "gnnfd_aggregate_workspace_bytes")
+    return s.value
+
+
+def _aggregate(fn, name, csr: Csr, x, f, chunk_width, out, out_dtype, scratch, stream):
+    f = x.shape[1] if f is None else f
+    chunk_width = f if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((csr.n, f), dtype=out_dtype or torch.float32, device=x.device)
+    xp, ldx = _matrix(x, f, "x")
+    op, ldo = _matrix(out, f, "out")
+    need = aggregate_workspace_bytes(csr, f)
+    if scratch is None and need:
+        scratch = _alloc_bytes(need, x.device)
+    sp = ctypes.c_void_p(scratch.data_ptr()) if scratch is not None else None
+    sn = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    _check(fn(csr.handle, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f, chunk_width, sp, sn,
+              _stream_ptr(stream)), name)
+    return out
+
+
+def aggregate_gcn(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width: int | None = None,
+                  out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None) -> torch.Tensor:
+    return _aggregate(lib().gnnfd_aggregate_gcn, "gnnfd_aggregate_gcn", csr, x, f, chunk_width, out, out_dtype,
+                      scratch, stream)
+
+
+def aggregate_sage(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width: int | None = None,
+                   out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None) -> torch.Tensor:
+    return _aggregate(lib().gnnfd_aggregate_sage, "gnnfd_aggregate_sage", csr, x, f, chunk_width, out, out_dtype,
+                      scratch, stream)
+
+
+def gat_scores(z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.Tensor, heads: int, dim: int, stream=None):
+    n = z.shape[0]
+    zp, ldz = _matrix(z, heads * dim, "z")
+    a_src = a_src.contiguous().float()
+    a_dst = a_dst.contiguous().float()
+    s_src = torch.empty((n, heads), dtype=torch.float32, device=z.device)
+    s_dst = torch.empty((n, heads), dtype=torch.float32, device=z.device)
+    _check(lib().gnnfd_gat_scores(n, zp, ldz, _dtype_code(z), ctypes.c_void_p(a_src.data_ptr()),
+                                  ctypes.c_void_p(a_dst.data_ptr()), heads, dim, ctypes.c_void_p(s_src.data_ptr()),
+                                  ctypes.c_void_p(s_dst.data_ptr()), _stream_ptr(stream)), "gnnfd_gat_scores")
+    return s_src, s_dst
+
+
+def gat_workspace_bytes(csr: Csr, heads: int, dim: int) -> int:
+    s = ctypes.c_size_t()
+    _check(lib().gnnfd_gat_workspace_bytes(csr.handle, heads, dim, ctypes.byref(s)), "gnnfd_gat_workspace_bytes")
+    return s.value
+
+
+def aggregate_gat(csr: Csr, z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.Tensor, heads: int, dim: int,
+                  negative_slope: float = 0.2, chunk_width: int | None = None, out: torch.Tensor | None = None,
+                  out_dtype=None, scratch=None, stream=None) -> torch.Tensor:
+    f = heads * dim
+    chunk_width = f if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((csr.n, f), dtype=out_dtype or torch.float32, device=z.device)
+    zp, ldz = _matrix(z, f, "z")
+    op, ldo = _matrix(out, f, "out")
+    a_src = a_src.contiguous().float()
+    a_dst = a_dst.contiguous().float()
+    if scratch is None:
+        scratch = _alloc_bytes(gat_workspace_bytes(csr, heads, dim), z.device)
+    _check(lib().gnnfd_aggregate_gat(csr.handle, zp, ldz, _dtype_code(z), ctypes.c_void_p(a_src.data_ptr()),
+                                     ctypes.c_void_p(a_dst.data_ptr()), heads, dim, negative_slope, op, ldo,
+                                     _dtype_code(out), chunk_width, ctypes.c_void_p(scratch.data_ptr()),
+                                     scratch.numel() * scratch.element_size(), _stream_ptr(stream)),
+           "gnnfd_aggregate_gat")
+    return out
+
+
+def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_slope: float = 0.2,
+                 out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    heads = s_src.shape[1]
+    s_src = s_src.contiguous()
+    s_dst = s_dst.contiguous()
+    if s_src.dtype != torch.float32 or s_dst.dtype != torch.float32 or s_src.shape != s_dst.shape:
+        raise TypeError("scores must be float32 [n, heads]")
+    if out is None:
+        out = torch.empty((csr.nnz, heads), dtype=torch.float32, device=s_src.device)
+    _check(lib().gnnfd_edge_softmax(csr.handle, ctypes.c_void_p(s_src.data_ptr()), ctypes.c_void_p(s_dst.data_ptr()),
+                                    heads, negative_slope, ctypes.c_void_p(out.data_ptr()), _stream_ptr(stream)),
+           "gnnfd_edge_softmax")
+    return out
+
+
+def launch_count() -> int:
+    return int(lib().gnnfd_launch_count())
+
+
+def kernel_timing_enable(on: bool = True):
+    _check(lib().gnnfd_kernel_timing_enable(int(on)), "gnnfd_kernel_timing_enable")
+
+
+def kernel_timing_read() -> dict:
+    """{kernel name: (total ms, launches)} since the last read."""
+    cap = 64
+    names = (ctypes.c_char_p * cap)()
+    ms = (ctypes.c_double * cap)()
+    cnt = (ctypes.c_int64 * cap)()
+    k = lib().gnnfd_kernel_timing_read(names, ms, cnt, cap)
+    if k < 0:
+        raise GnnfdError(k, "gnnfd_kernel_timing_read")
+    return {names[i].decode(): (ms[i], cnt[i]) for i in range(min(k, cap))}

@@ -1,0 +1,315 @@
+// Chunked gather-aggregate for GCN and GraphSAGE (Algorithm 1: Message + Aggregate per decomposition
+// layer, Concat by writing each chunk into its own output columns) and the second-level reduction
+// of hub rows.
+//
+// Work decomposition.  One launch sweeps the chunks one after the other (the block index is
+// chunk-major), so at any time the blocks in flight gather from one chunk's n x chunk_width slice of
+// x, which is what keeps the gathered working set small enough for L2.  Inside a sweep the rows come
+// grouped by degree class.  A row is owned by S = LPR * EP lanes: LPR lanes cover the chunk's columns
+// with one 16-byte vector each, and EP groups of LPR lanes walk interleaved edges of the row, each
+// keeping U loads in flight.  The EP partial sums are combined by a fixed shuffle tree, hub rows
+// (degree > GNNFD_HUB_DEGREE) by per-segment partial sums that a second kernel adds in ascending
+// segment order: no atomics, bit-identical from run to run.
+#include <cuda_bf16.h>
+
+#include "schedule.cuh"
+
+namespace gnnfd {
+
+struct GatherArgs {
+    const int32_t* row_ptr;
+    const int32_t* col_idx;
+    const float* edge_w;
+    const float* rdeg;
+    const int32_t* row_order;
+    const int32_t* seg_row;
+    const int32_t* seg_begin;
+    const void* x;
+    void* out;
+    float* partial;
+    int64_t ldx, ldo;
+    int32_t f, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16, out_vec_ok;
+    int32_t n_ranges;
+    Range range[kMaxRanges];
+};
+
+// ---- per-lane vectors: VECN elements of T, widened to fp32
+
+template <typename T, int VECN> struct Vec;
+
+template <> struct Vec<float, 4> {
+    float4 v;
+    __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
+    __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
+    __device__ __forceinline__ float get(int i) const { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+};
+template <> struct Vec<float, 1> {
+    float v;
+    __device__ __forceinline__ void load(const float* p) { v = __ldg(p); }
+    __device__ __forceinline__ void zero() { v = 0.f; }
+    __device__ __forceinline__ float get(int) const { return v; }
+};
+template <> struct Vec<__nv_bfloat16, 8> {
+    uint4 v;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint4*>(p)); }
+    __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ float get(int i) const
+    {
+        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
+        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));   // bf16 -> fp32 is exact
+    }
+};
+template <> struct Vec<__nv_bfloat16, 1> {
+    unsigned short v;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const unsigned short*>(p)); }
+    __device__ __forceinline__ void zero() { v = 0; }
+    __device__ __forceinline__ float get(int) const { return __uint_as_float((uint32_t)v << 16); }
+};
+
+__device__ __forceinline__ void store_elem(void* out, int out_bf16, int64_t idx, float val)
+{
+    if (out_bf16) static_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(val);
+    else __stcs(static_cast<float*>(out) + idx, val);
+}
+
+// One row (or hub segment) per S = LPR * EP lanes.
+template <typename T, int VECN, int LPR, bool WEIGHTED, int EP>
+__device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0,
+                                            int chunk_end)
+{
+    constexpr int S = LPR * EP;
+    constexpr int ROWS = kBlock / S;
+    const int tid = threadIdx.x;
+    const int slot = block_in_range * ROWS + tid / S;
+    const int ls = tid % S;
+    const int g = ls / LPR;
+    const int j = col0 + (ls % LPR) * VECN;
+    const bool col_ok = j < chunk_end;
+    const bool active = slot < rg.item_count;
+
+    int32_t row = 0, b = 0, e = 0;
+    if (active) {
+        if (rg.hub) {
+            row = a.seg_row[slot];
+            b = a.seg_begin[slot];
+            e = min(b + kHubSegment, a.row_ptr[row + 1]);
+        } else {
+            row = a.row_order[rg.item_begin + slot];
+            b = a.row_ptr[row];
+            e = a.row_ptr[row + 1];
+        }
+    }
+
+    float acc[VECN];
+#pragma unroll
+    for (int i = 0; i < VECN; ++i) acc[i] = 0.f;
+    const T* xj = static_cast<const T*>(a.x) + j;
+
+    for (int32_t k = b + g; k < e; k += EP * kUnroll) {
+        int32_t u[kUnroll];
+        float w[kUnroll];
+#pragma unroll
+        for (int t = 0; t < kUnroll; ++t) {
+            const int32_t kk = k + t * EP;
+            const bool ok = kk < e;
+            u[t] = ok ? __ldcs(a.col_idx + kk) : -1;
+            if (WEIGHTED) w[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
+        }
+        Vec<T, VECN> v[kUnroll];
+#pragma unroll
+        for (int t = 0; t < kUnroll; ++t) {
+            if (u[t] >= 0 && col_ok) v[t].load(xj + (int64_t)u[t] * a.ldx);
+            else v[t].zero();
+        }
+#pragma unroll
+        for (int t = 0; t < kUnroll; ++t) {
+#pragma unroll
+            for (int i = 0; i < VECN; ++i) {
+                if (WEIGHTED) acc[i] = fmaf(w[t], v[t].get(i), acc[i]);
+                else acc[i] += v[t].get(i);
+            }
+        }
+    }
+
+    // fixed-order combination of the EP partial sums of the row
+#pragma unroll
+    for (int o = S / 2; o >= LPR; o >>= 1) {
+#pragma unroll
+        for (int i = 0; i < VECN; ++i) acc[i] += __shfl_down_sync(0xffffffffu, acc[i], o, S);
+    }
+
+    if (!active || g != 0 || !col_ok) return;
+    if (rg.hub) {
+        float* p = a.partial + (int64_t)slot * a.fpad + j;
+#pragma unroll
+        for (int i = 0; i < VECN; ++i)
+            if (j + i < chunk_end) p[i] = acc[i];
+        return;
+    }
+    const float scale = WEIGHTED ? 1.f : a.rdeg[row];
+    const int64_t o = (int64_t)row * a.ldo + j;
+    if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
+#pragma unroll
+        for (int i = 0; i < VECN; i += 4)
+            __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
+                   make_float4(acc[i] * scale, acc[i + 1] * scale, acc[i + 2] * scale, acc[i + 3] * scale));
+    } else {
+#pragma unroll
+        for (int i = 0; i < VECN; ++i)
+            if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[i] * scale);
+    }
+}
+
+template <typename T, int VECN, int LPR, bool WEIGHTED>
+__global__ void __launch_bounds__(kBlock) gather_aggregate(const __grid_constant__ GatherArgs a)
+{
+    const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
+    const int chunk = (int)(blockIdx.x / per_chunk);
+    const int rem = (int)(blockIdx.x % per_chunk);
+    const int rb = rem / a.n_ctiles;
+    const int ctile = rem % a.n_ctiles;
+    const int chunk_begin = chunk * a.chunk_width;
+    const int chunk_end = min(a.f, chunk_begin + a.chunk_width);
+    const int col0 = chunk_begin + ctile * (LPR * VECN);
+    if (col0 >= chunk_end) return;
+    int r = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxRanges; ++i)
+        if (i < a.n_ranges && rb >= a.range[i].first_block) r = i;
+    const Range rg = a.range[r];
+    const int bir = rb - rg.first_block;
+    switch (rg.ep_log2) {
+        case 0: gather_rows<T, VECN, LPR, WEIGHTED, 1>(a, rg, bir, col0, chunk_end); break;
+        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 2>(a, rg, bir, col0, chunk_end); break;
+        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 4>(a, rg, bir, col0, chunk_end); break;
+        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 8>(a, rg, bir, col0, chunk_end); break;
+        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 16>(a, rg, bir, col0, chunk_end); break;
+        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, WEIGHTED, 32>(a, rg, bir, col0, chunk_end); break;
+    }
+}
+
+// out[row, j] = scale * sum over the row's segments, ascending, of partial[segment, j]
+__global__ void __launch_bounds__(kBlock)
+hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict__ hub_seg_ptr, const float* __restrict__ rdeg,
+           const float* __restrict__ partial, int64_t hub_begin, int32_t n_hub, int32_t f, int32_t fpad, int use_rdeg,
+           void* __restrict__ out, int64_t ldo, int out_bf16)
+{
+    const int i = blockIdx.x;
+    const int j = blockIdx.y * kBlock + threadIdx.x;
+    if (i >= n_hub || j >= f) return;
+    const int32_t row = row_order[hub_begin + i];
+    const int32_t s0 = hub_seg_ptr[i], s1 = hub_seg_ptr[i + 1];
+    float acc = 0.f;
+    for (int32_t s = s0; s < s1; ++s) acc += partial[(int64_t)s * fpad + j];
+    if (use_rdeg) acc *= rdeg[row];
+    store_elem(out, out_bf16, (int64_t)row * ldo + j, acc);
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef void (*GatherKernel)(const GatherArgs);
+
+template <typename T, int VECN, bool WEIGHTED>
+static GatherKernel pick_lpr(int lpr)
+{
+    switch (lpr) {
+        case 1: return gather_aggregate<T, VECN, 1, WEIGHTED>;
+        case 2: return gather_aggregate<T, VECN, 2, WEIGHTED>;
+        case 4: return gather_aggregate<T, VECN, 4, WEIGHTED>;
+        case 8: return gather_aggregate<T, VECN, 8, WEIGHTED>;
+        case 16: return gather_aggregate<T, VECN, 16, WEIGHTED>;
+        default: return gather_aggregate<T, VECN, 32, WEIGHTED>;
+    }
+}
+
+template <bool WEIGHTED>
+static GatherKernel pick_kernel(gnnfd_dtype_t xdt, bool vec, int lpr)
+{
+    if (xdt == GNNFD_F32) return vec ? pick_lpr<float, 4, WEIGHTED>(lpr) : pick_lpr<float, 1, WEIGHTED>(lpr);
+    return vec ? pick_lpr<__nv_bfloat16, 8, WEIGHTED>(lpr) : pick_lpr<__nv_bfloat16, 1, WEIGHTED>(lpr);
+}
+
+static size_t partial_bytes(const gnnfd_csr_t* csr, int32_t f)
+{
+    const size_t fpad = align_up((size_t)f, 4);
+    return align_up((size_t)csr->n_segments * fpad * sizeof(float), 256);
+}
+
+static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out,
+                     int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width, void* d_scratch,
+                     size_t scratch_bytes, cudaStream_t s)
+{
+    if (!csr || !d_x || !d_out || f <= 0 || chunk_width <= 0 || ldx < f || ldo < f) return GNNFD_INVALID_ARG;
+    if ((xdt != GNNFD_F32 && xdt != GNNFD_BF16) || (odt != GNNFD_F32 && odt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
+    const size_t need = partial_bytes(csr, f);
+    if (need > 0 && (!d_scratch || scratch_bytes < need)) return GNNFD_WORKSPACE_TOO_SMALL;
+    if (need > 0 && ((uintptr_t)d_scratch & 15u)) return GNNFD_INVALID_ARG;
+
+    const int cw = chunk_width < f ? chunk_width : f;
+    const int n_chunks = (f + cw - 1) / cw;
+    const int xsize = xdt == GNNFD_F32 ? 4 : 2;
+    const int vecn = 16 / xsize;
+    // 128-bit loads need 16-byte aligned row starts and chunk starts
+    const bool vec = ((uintptr_t)d_x % 16 == 0) && ((ldx * xsize) % 16 == 0) && (n_chunks == 1 || cw % vecn == 0);
+    const int elems = vec ? vecn : 1;
+    int lanes = (cw + elems - 1) / elems;
+    int lpr = 1;
+    while (lpr < lanes && lpr < 32) lpr <<= 1;
+
+    GatherArgs a;
+    a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.edge_w = csr->edge_w; a.rdeg = csr->rdeg;
+    a.row_order = csr->row_order; a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin;
+    a.x = d_x; a.out = d_out; a.partial = static_cast<float*>(d_scratch);
+    a.ldx = ldx; a.ldo = ldo; a.f = f; a.chunk_width = cw;
+    a.n_ctiles = (cw + lpr * elems - 1) / (lpr * elems);
+    a.fpad = (int32_t)align_up((size_t)f, 4);
+    a.out_bf16 = odt == GNNFD_BF16;
+    a.out_vec_ok = odt == GNNFD_F32 && ((uintptr_t)d_out % 16 == 0) && (ldo % 4 == 0) && (n_chunks == 1 || cw % 4 == 0);
+
+    const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges);
+    a.blocks_per_tile = (int32_t)blocks;
+    const int64_t grid = blocks * a.n_ctiles * n_chunks;
+    if (grid > 0x7fffffffll || blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
+
+    if (grid > 0) {
+        GatherKernel kernel = weighted ? pick_kernel<true>(xdt, vec, lpr) : pick_kernel<false>(xdt, vec, lpr);
+        GNNFD_LAUNCH(weighted ? "gather_aggregate_gcn" : "gather_aggregate_sage", s, kernel, (unsigned)grid, kBlock, 0, a);
+    }
+    const int64_t n_hub = csr->bin_count[4];
+    if (n_hub > 0) {
+        dim3 g((unsigned)n_hub, (unsigned)((f + kBlock - 1) / kBlock));
+        GNNFD_LAUNCH("hub_reduce", s, hub_reduce, g, kBlock, 0, csr->row_order, csr->hub_seg_ptr, csr->rdeg, a.partial,
+                     csr->bin_start[4], (int32_t)n_hub, f, a.fpad, weighted ? 0 : 1, d_out, ldo, a.out_bf16);
+    }
+    GNNFD_CUDA_CHECK(cudaGetLastError());
+    return GNNFD_OK;
+}
+
+}  // namespace gnnfd
+
+extern "C" {
+
+int gnnfd_aggregate_workspace_bytes(const gnnfd_csr_t* csr, int32_t f, size_t* scratch_bytes)
+{
+    if (!csr || f <= 0 || !scratch_bytes) return GNNFD_INVALID_ARG;
+    *scratch_bytes = gnnfd::partial_bytes(csr, f);
+    return GNNFD_OK;
+}
+
+int gnnfd_aggregate_gcn(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out, int64_t ldo,
+                        gnnfd_dtype_t odt, int32_t f, int32_t chunk_width, void* d_scratch, size_t scratch_bytes,
+                        void* stream)
+{
+    return gnnfd::aggregate(true, csr, d_x, ldx, xdt, d_out, ldo, odt, f, chunk_width, d_scratch, scratch_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int gnnfd_aggregate_sage(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out, int64_t ldo,
+                         gnnfd_dtype_t odt, int32_t f, int32_t chunk_width, void* d_scratch, size_t scratch_bytes,
+                         void* stream)
+{
+    return gnnfd::aggregate(false, csr, d_x, ldx, xdt, d_out, ldo, odt, f, chunk_width, d_scratch, scratch_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,509 @@
+// Device CSR-by-destination builder: key generation, stable LSD radix sort of (dst, src) keys,
+// duplicate removal, row pointers, degree normalisers, GCN edge weights and the launch schedule
+// (degree bins, hub segments).  Integer work throughout; the only host synchronisation is the
+// final read of the counters.
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace gnnfd {
+
+using u64 = unsigned long long;
+
+constexpr int kThreads = 256;
+constexpr int kRadixBits = 8;
+constexpr int kRadix = 1 << kRadixBits;
+constexpr int kSortItems = 16;                       // keys per thread
+constexpr int kSortTile = kThreads * kSortItems;     // keys per block
+constexpr int kSortWarps = kThreads / 32;
+constexpr int kWarpItems = 32 * kSortItems;
+
+static inline unsigned blocks_for(size_t count, int per_block)
+{
+    size_t b = (count + per_block - 1) / per_block;
+    return (unsigned)(b ? b : 1);
+}
+
+// ------------------------------------------------------------------ keys
+
+// Candidate i < e: input edge i.  e <= i < 2e (symmetrise): reverse of edge i - e.  Then one
+// self-loop per vertex (value -1).  Dropped candidates get the key 1 << (2*bits), above every
+// valid key, so the sort moves them behind the kept ones.
+template <typename IdT>
+__global__ void __launch_bounds__(kThreads)
+make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, int64_t e, int64_t m, uint32_t flags,
+          int bits, u64* __restrict__ keys, int32_t* __restrict__ vals, BuildCounts* __restrict__ counts)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const u64 invalid = 1ull << (2 * bits);
+    const int64_t n_rev = (flags & GNNFD_CSR_SYMMETRIZE) ? e : 0;
+    bool keep = false, bad = false;
+    if (i < m) {
+        int64_t s, d;
+        int32_t val;
+        if (i < e) {
+            s = (int64_t)src[i]; d = (int64_t)dst[i]; val = (int32_t)i;
+            bad = s < 0 || s >= n || d < 0 || d >= n;
+            keep = !bad && !((flags & GNNFD_CSR_ADD_SELF_LOOPS) && s == d);
+        } else if (i < e + n_rev) {
+            s = (int64_t)dst[i - e]; d = (int64_t)src[i - e]; val = (int32_t)i;
+            keep = !(s < 0 || s >= n || d < 0 || d >= n) && s != d;
+        } else {
+            s = d = i - e - n_rev; val = -1;
+            keep = true;
+        }
+        keys[i] = keep ? (((u64)d << bits) | (u64)s) : invalid;
+        vals[i] = val;
+    }
+    const unsigned kept = __ballot_sync(0xffffffffu, keep);
+    const unsigned bads = __ballot_sync(0xffffffffu, bad);
+    if ((threadIdx.x & 31) == 0) {
+        if (kept) atomicAdd(&counts->n_valid, __popc(kept));
+        if (bads) atomicAdd(&counts->bad_index, __popc(bads));
+    }
+}
+
+// ------------------------------------------------------------------ radix sort (one 8-bit digit per pass)
+
+__global__ void __launch_bounds__(kThreads)
+radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int64_t n_tiles, int32_t* __restrict__ hist)
+{
+    __shared__ int32_t h[kRadix];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kSortTile;
+#pragma unroll
+    for (int i = 0; i < kSortItems; ++i) {
+        const int64_t idx = base + i * kThreads + threadIdx.x;
+        if (idx < m) atomicAdd(&h[(int)((keys[idx] >> shift) & (kRadix - 1))], 1);
+    }
+    __syncthreads();
+    hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
+}
+
+// Stable scatter.  A warp owns 512 consecutive keys of the tile and walks them 32 at a time; keys
+// with equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp
+// running count, across warps by a prefix over the per-warp counts, across tiles by the scanned
+// histogram.
+__global__ void __launch_bounds__(kThreads)
+radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_in, u64* __restrict__ keys_out,
+              int32_t* __restrict__ vals_out, int64_t m, int shift, int64_t n_tiles,
+              const int32_t* __restrict__ tile_offset)
+{
+    __shared__ int32_t warp_count[kSortWarps][kRadix];
+    __shared__ int32_t global_base[kRadix];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) warp_count[w][threadIdx.x] = 0;
+    __syncthreads();
+
+    const int64_t warp_base = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * kWarpItems;
+    u64 key[kSortItems];
+    int32_t rank[kSortItems];
+#pragma unroll
+    for (int r = 0; r < kSortItems; ++r) {
+        const int64_t idx = warp_base + r * 32 + lane;
+        const bool valid = idx < m;
+        key[r] = valid ? keys_in[idx] : 0ull;
+        const int digit = valid ? (int)((key[r] >> shift) & (kRadix - 1)) : kRadix;
+        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        const int leader = __ffs(peers) - 1;
+        int32_t before = 0;
+        if (lane == leader && valid) {
+            before = warp_count[warp][digit];
+            warp_count[warp][digit] = before + __popc(peers);
+        }
+        before = __shfl_sync(0xffffffffu, before, leader);
+        rank[r] = before + __popc(peers & ((1u << lane) - 1u));
+        __syncwarp();
+    }
+    __syncthreads();
+    {
+        int32_t run = 0;
+#pragma unroll
+        for (int w = 0; w < kSortWarps; ++w) {
+            const int32_t c = warp_count[w][threadIdx.x];
+            warp_count[w][threadIdx.x] = run;
+            run += c;
+        }
+        global_base[threadIdx.x] = tile_offset[(int64_t)threadIdx.x * n_tiles + blockIdx.x];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kSortItems; ++r) {
+        const int64_t idx = warp_base + r * 32 + lane;
+        if (idx < m) {
+            const int digit = (int)((key[r] >> shift) & (kRadix - 1));
+            const int64_t pos = (int64_t)global_base[digit] + warp_count[warp][digit] + rank[r];
+            keys_out[pos] = key[r];
+            vals_out[pos] = vals_in[idx];
+        }
+    }
+}
+
+// ------------------------------------------------------------------ after the sort
+
+// flag[i] = 1 for the first of each run of equal keys among the kept candidates
+__global__ void __launch_bounds__(kThreads)
+flag_first_of_run(const u64* __restrict__ keys, int64_t m, const BuildCounts* __restrict__ counts,
+                  int32_t* __restrict__ flag)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= m) return;
+    flag[i] = (i < counts->n_valid && (i == 0 || keys[i] != keys[i - 1])) ? 1 : 0;
+}
+
+__global__ void __launch_bounds__(kThreads)
+compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const int32_t* __restrict__ flag,
+               const int32_t* __restrict__ pos, int64_t m, u64* __restrict__ keys_out, int32_t* __restrict__ perm,
+               BuildCounts* __restrict__ counts)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= m) return;
+    if (flag[i]) {
+        keys_out[pos[i]] = keys[i];
+        perm[pos[i]] = vals[i];
+    }
+    if (i == m - 1) counts->nnz = pos[i] + flag[i];
+}
+
+__global__ void __launch_bounds__(kThreads)
+copy_perm(const int32_t* __restrict__ vals, int64_t m, int32_t* __restrict__ perm, BuildCounts* __restrict__ counts)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (i == 0) counts->nnz = counts->n_valid;
+    if (i < m && i < counts->n_valid) perm[i] = vals[i];
+}
+
+// row_ptr[v] = number of kept keys with dst < v (binary search in the sorted keys)
+__global__ void __launch_bounds__(kThreads)
+row_pointers(const u64* __restrict__ keys, const BuildCounts* __restrict__ counts, int64_t n, int bits,
+             int32_t* __restrict__ row_ptr)
+{
+    const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (v > n) return;
+    const u64 target = (u64)v << bits;
+    int32_t lo = 0, hi = counts->nnz;
+    while (lo < hi) {
+        const int32_t mid = lo + ((hi - lo) >> 1);
+        if (keys[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    row_ptr[v] = lo;
+}
+
+__device__ __forceinline__ int degree_bin(int32_t deg)
+{
+    return deg <= kBinDeg0 ? 0 : deg <= kBinDeg1 ? 1 : deg <= kBinDeg2 ? 2 : deg <= kBinDeg3 ? 3 : 4;
+}
+
+// degree normalisers (rounded once from fp64) and the bin membership flags, bin-major [5][n]
+__global__ void __launch_bounds__(kThreads)
+degrees_and_bins(const int32_t* __restrict__ row_ptr, int64_t n, float* __restrict__ dinv, float* __restrict__ rdeg,
+                 int32_t* __restrict__ bin_flag, BuildCounts* __restrict__ counts)
+{
+    const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    int32_t deg = 0;
+    if (v < n) {
+        deg = row_ptr[v + 1] - row_ptr[v];
+        dinv[v] = deg > 0 ? (float)(1.0 / sqrt((double)deg)) : 0.f;
+        rdeg[v] = deg > 0 ? (float)(1.0 / (double)deg) : 0.f;
+        const int bin = degree_bin(deg);
+#pragma unroll
+        for (int b = 0; b < kNumBins; ++b) bin_flag[(int64_t)b * n + v] = b == bin ? 1 : 0;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) deg = max(deg, __shfl_xor_sync(0xffffffffu, deg, o));
+    if ((threadIdx.x & 31) == 0 && deg > 0) atomicMax(&counts->max_degree, deg);
+}
+
+// col_idx and the GCN weight of every slot, from the sorted keys
+__global__ void __launch_bounds__(kThreads)
+columns_and_weights(const u64* __restrict__ keys, const BuildCounts* __restrict__ counts, int bits,
+                    const float* __restrict__ dinv, int32_t* __restrict__ col_idx, float* __restrict__ edge_w, int64_t m)
+{
+    const int64_t k = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (k >= m || k >= counts->nnz) return;
+    const u64 key = keys[k];
+    const int32_t s = (int32_t)(key & ((1ull << bits) - 1ull));
+    const int32_t d = (int32_t)(key >> bits);
+    col_idx[k] = s;
+    edge_w[k] = dinv[s] * dinv[d];
+}
+
+__global__ void __launch_bounds__(kThreads)
+place_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ bin_pos, int64_t n,
+           int32_t* __restrict__ row_order, BuildCounts* __restrict__ counts)
+{
+    const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (v < n) {
+        const int bin = degree_bin(row_ptr[v + 1] - row_ptr[v]);
+        row_order[bin_pos[(int64_t)bin * n + v]] = (int32_t)v;
+    }
+    if (v == 0) {
+        for (int b = 0; b < kNumBins; ++b) {
+            const int32_t start = bin_pos[(int64_t)b * n];
+            const int32_t end = b + 1 < kNumBins ? bin_pos[(int64_t)(b + 1) * n] : (int32_t)n;
+            counts->bin_count[b] = end - start;
+        }
+    }
+}
+
+// segments per hub row; entry n_hub (one past the end) is 0 so that the scan yields the total
+__global__ void __launch_bounds__(kThreads)
+hub_segment_counts(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ row_order, int64_t n,
+                   const BuildCounts* __restrict__ counts, int64_t hub_cap, int32_t* __restrict__ seg_count)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (i > hub_cap) return;
+    const int32_t n_hub = counts->bin_count[4];
+    int32_t c = 0;
+    if (i < n_hub) {
+        const int32_t v = row_order[n - n_hub + i];
+        c = (row_ptr[v + 1] - row_ptr[v] + kHubSegment - 1) / kHubSegment;
+    }
+    seg_count[i] = c;
+}
+
+__global__ void __launch_bounds__(kThreads)
+fill_segments(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ row_order, int64_t n,
+              BuildCounts* __restrict__ counts, const int32_t* __restrict__ hub_seg_ptr, int64_t hub_cap,
+              int32_t* __restrict__ seg_row, int32_t* __restrict__ seg_begin)
+{
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const int32_t n_hub = counts->bin_count[4];
+    if (i == 0) counts->n_segments = hub_seg_ptr[n_hub];
+    if (i >= hub_cap || i >= n_hub) return;
+    const int32_t v = row_order[n - n_hub + i];
+    const int32_t b = row_ptr[v];
+    const int32_t first = hub_seg_ptr[i], last = hub_seg_ptr[i + 1];
+    for (int32_t s = first; s < last; ++s) {
+        seg_row[s] = v;
+        seg_begin[s] = b + (s - first) * kHubSegment;
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+struct BuildLayout {
+    int64_t m;             // candidate edges
+    int64_t n_tiles;       // sort tiles
+    int64_t hub_cap;       // upper bound on hub rows
+    int64_t seg_cap;       // upper bound on hub segments
+    int bits, key_bits, passes;
+};
+
+static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
+{
+    if (n <= 0 || e < 0) return GNNFD_INVALID_ARG;
+    if (flags & ~(uint32_t)(GNNFD_CSR_ADD_SELF_LOOPS | GNNFD_CSR_DEDUP | GNNFD_CSR_SYMMETRIZE)) return GNNFD_INVALID_ARG;
+    const int64_t limit = (int64_t(1) << 31) - 1;
+    if (n > limit || e > limit) return GNNFD_TOO_LARGE;
+    int64_t m = e;
+    if (flags & GNNFD_CSR_SYMMETRIZE) m += e;
+    if (flags & GNNFD_CSR_ADD_SELF_LOOPS) m += n;
+    if (m > limit) return GNNFD_TOO_LARGE;
+    L->m = m;
+    L->n_tiles = (m + kSortTile - 1) / kSortTile;
+    if (L->n_tiles == 0) L->n_tiles = 1;
+    L->hub_cap = m / (GNNFD_HUB_DEGREE + 1) + 1;
+    L->seg_cap = m / kHubSegment + L->hub_cap + 1;
+    int bits = 1;
+    while ((int64_t(1) << bits) < n) ++bits;
+    L->bits = bits;
+    L->key_bits = 2 * bits + 1;
+    L->passes = (L->key_bits + kRadixBits - 1) / kRadixBits;
+    return GNNFD_OK;
+}
+
+struct PersistentPtrs {
+    int32_t *row_ptr, *col_idx, *perm, *row_order, *seg_row, *seg_begin, *hub_seg_ptr;
+    float *edge_w, *dinv, *rdeg;
+    BuildCounts* counts;
+};
+
+static void carve_persistent(Carver& c, int64_t n, const BuildLayout& L, PersistentPtrs* p)
+{
+    const size_t cap = (size_t)(L.m > 0 ? L.m : 1);
+    p->row_ptr = c.take<int32_t>((size_t)n + 1);
+    p->col_idx = c.take<int32_t>(cap);
+    p->perm = c.take<int32_t>(cap);
+    p->edge_w = c.take<float>(cap);
+    p->dinv = c.take<float>((size_t)n);
+    p->rdeg = c.take<float>((size_t)n);
+    p->row_order = c.take<int32_t>((size_t)n);
+    p->seg_row = c.take<int32_t>((size_t)L.seg_cap);
+    p->seg_begin = c.take<int32_t>((size_t)L.seg_cap);
+    p->hub_seg_ptr = c.take<int32_t>((size_t)L.hub_cap + 1);
+    p->counts = c.take<BuildCounts>(1);
+}
+
+struct ScratchPtrs {
+    u64 *keys_a, *keys_b;
+    int32_t *vals_a, *vals_b, *hist, *flags, *scan_temp;
+};
+
+static size_t flag_ints(int64_t n, const BuildLayout& L)
+{
+    size_t a = (size_t)L.m, b = (size_t)kNumBins * (size_t)n, c = (size_t)L.hub_cap + 1;
+    size_t r = a > b ? a : b;
+    return (r > c ? r : c) + 1;
+}
+
+static void carve_scratch(Carver& c, int64_t n, const BuildLayout& L, ScratchPtrs* p)
+{
+    const size_t cap = (size_t)(L.m > 0 ? L.m : 1);
+    p->keys_a = c.take<u64>(cap);
+    p->keys_b = c.take<u64>(cap);
+    p->vals_a = c.take<int32_t>(cap);
+    p->vals_b = c.take<int32_t>(cap);
+    const size_t hist_ints = (size_t)kRadix * (size_t)L.n_tiles;
+    p->hist = c.take<int32_t>(hist_ints);
+    const size_t fl = flag_ints(n, L);
+    p->flags = c.take<int32_t>(fl);
+    const size_t biggest = hist_ints > fl ? hist_ints : fl;
+    p->scan_temp = c.take<int32_t>(scan_temp_ints(biggest));
+}
+
+}  // namespace gnnfd
+
+extern "C" {
+
+int gnnfd_csr_workspace_bytes(int64_t n, int64_t e, uint32_t flags, size_t* persistent_bytes, size_t* scratch_bytes)
+{
+    using namespace gnnfd;
+    BuildLayout L;
+    int rc = make_layout(n, e, flags, &L);
+    if (rc) return rc;
+    if (persistent_bytes) {
+        Carver c(nullptr, ~size_t(0));
+        PersistentPtrs p;
+        carve_persistent(c, n, L, &p);
+        *persistent_bytes = c.off;
+    }
+    if (scratch_bytes) {
+        Carver c(nullptr, ~size_t(0));
+        ScratchPtrs s;
+        carve_scratch(c, n, L, &s);
+        *scratch_bytes = c.off;
+    }
+    return GNNFD_OK;
+}
+
+int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, gnnfd_itype_t itype, uint32_t flags,
+                    void* d_persistent, size_t persistent_bytes, void* d_scratch, size_t scratch_bytes, void* stream,
+                    gnnfd_csr_t** out)
+{
+    using namespace gnnfd;
+    if (!out) return GNNFD_INVALID_ARG;
+    *out = nullptr;
+    BuildLayout L;
+    int rc = make_layout(n, e, flags, &L);
+    if (rc) return rc;
+    if (itype != GNNFD_I32 && itype != GNNFD_I64) return GNNFD_UNSUPPORTED;
+    if ((e > 0 && (!d_src || !d_dst)) || !d_persistent || !d_scratch) return GNNFD_INVALID_ARG;
+    if (((uintptr_t)d_persistent | (uintptr_t)d_scratch) & 255u) return GNNFD_INVALID_ARG;
+
+    Carver pc(d_persistent, persistent_bytes), sc(d_scratch, scratch_bytes);
+    PersistentPtrs P;
+    ScratchPtrs S;
+    carve_persistent(pc, n, L, &P);
+    carve_scratch(sc, n, L, &S);
+    if (!pc.ok || !sc.ok) return GNNFD_WORKSPACE_TOO_SMALL;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t m = L.m;
+    GNNFD_CUDA_CHECK(cudaMemsetAsync(P.counts, 0, sizeof(BuildCounts), s));
+
+    BuildCounts host_counts;
+    std::memset(&host_counts, 0, sizeof(host_counts));
+    u64* keys = S.keys_a;
+    u64* keys_alt = S.keys_b;
+    int32_t* vals = S.vals_a;
+    int32_t* vals_alt = S.vals_b;
+
+    if (m > 0) {
+        if (itype == GNNFD_I32)
+            GNNFD_LAUNCH("make_keys", s, make_keys<int32_t>, blocks_for(m, kThreads), kThreads, 0,
+                         static_cast<const int32_t*>(d_src), static_cast<const int32_t*>(d_dst), n, e, m, flags, L.bits,
+                         keys, vals, P.counts);
+        else
+            GNNFD_LAUNCH("make_keys", s, make_keys<long long>, blocks_for(m, kThreads), kThreads, 0,
+                         static_cast<const long long*>(d_src), static_cast<const long long*>(d_dst), n, e, m, flags,
+                         L.bits, keys, vals, P.counts);
+        for (int pass = 0; pass < L.passes; ++pass) {
+            const int shift = pass * kRadixBits;
+            GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.n_tiles, kThreads, 0, keys, m, shift,
+                         L.n_tiles, S.hist);
+            rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.n_tiles, S.scan_temp, s);
+            if (rc) return rc;
+            GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.n_tiles, kThreads, 0, keys, vals, keys_alt,
+                         vals_alt, m, shift, L.n_tiles, S.hist);
+            u64* tk = keys; keys = keys_alt; keys_alt = tk;
+            int32_t* tv = vals; vals = vals_alt; vals_alt = tv;
+        }
+        if (flags & GNNFD_CSR_DEDUP) {
+            GNNFD_LAUNCH("flag_first_of_run", s, flag_first_of_run, blocks_for(m, kThreads), kThreads, 0, keys, m,
+                         P.counts, S.flags);
+            int32_t* pos = vals_alt;   // free after the last pass
+            rc = exclusive_scan_i32(S.flags, pos, (size_t)m, S.scan_temp, s);
+            if (rc) return rc;
+            GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys, vals, S.flags,
+                         pos, m, keys_alt, P.perm, P.counts);
+            keys = keys_alt;
+        } else {
+            GNNFD_LAUNCH("copy_perm", s, copy_perm, blocks_for(m, kThreads), kThreads, 0, vals, m, P.perm, P.counts);
+        }
+    }
+    GNNFD_LAUNCH("row_pointers", s, row_pointers, blocks_for((size_t)n + 1, kThreads), kThreads, 0, keys, P.counts, n,
+                 L.bits, P.row_ptr);
+    GNNFD_LAUNCH("degrees_and_bins", s, degrees_and_bins, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
+                 P.dinv, P.rdeg, S.flags, P.counts);
+    if (m > 0)
+        GNNFD_LAUNCH("columns_and_weights", s, columns_and_weights, blocks_for(m, kThreads), kThreads, 0, keys, P.counts,
+                     L.bits, P.dinv, P.col_idx, P.edge_w, m);
+    rc = exclusive_scan_i32(S.flags, S.flags, (size_t)kNumBins * (size_t)n, S.scan_temp, s);
+    if (rc) return rc;
+    GNNFD_LAUNCH("place_rows", s, place_rows, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, S.flags, n,
+                 P.row_order, P.counts);
+    // the bin positions are consumed; reuse the flag buffer for the per-hub-row segment counts
+    int32_t* seg_count = S.flags;
+    GNNFD_LAUNCH("hub_segment_counts", s, hub_segment_counts, blocks_for((size_t)L.hub_cap + 1, kThreads), kThreads, 0,
+                 P.row_ptr, P.row_order, n, P.counts, L.hub_cap, seg_count);
+    rc = exclusive_scan_i32(seg_count, P.hub_seg_ptr, (size_t)L.hub_cap + 1, S.scan_temp, s);
+    if (rc) return rc;
+    GNNFD_LAUNCH("fill_segments", s, fill_segments, blocks_for((size_t)L.hub_cap, kThreads), kThreads, 0, P.row_ptr,
+                 P.row_order, n, P.counts, P.hub_seg_ptr, L.hub_cap, P.seg_row, P.seg_begin);
+    GNNFD_CUDA_CHECK(cudaGetLastError());
+    GNNFD_CUDA_CHECK(cudaMemcpyAsync(&host_counts, P.counts, sizeof(BuildCounts), cudaMemcpyDeviceToHost, s));
+    GNNFD_CUDA_CHECK(cudaStreamSynchronize(s));
+
+    if (host_counts.bad_index > 0) return GNNFD_BAD_INDEX;
+
+    gnnfd_csr_t* h = new (std::nothrow) gnnfd_csr_t;
+    if (!h) return GNNFD_INVALID_ARG;
+    h->n = n;
+    h->nnz = host_counts.nnz;
+    h->max_degree = host_counts.max_degree;
+    int64_t start = 0;
+    for (int b = 0; b < kNumBins; ++b) {
+        h->bin_count[b] = host_counts.bin_count[b];
+        h->bin_start[b] = start;
+        start += host_counts.bin_count[b];
+    }
+    h->n_segments = host_counts.n_segments;
+    h->row_ptr = P.row_ptr;
+    h->col_idx = P.col_idx;
+    h->perm = P.perm;
+    h->dinv = P.dinv;
+    h->rdeg = P.rdeg;
+    h->edge_w = P.edge_w;
+    h->row_order = P.row_order;
+    h->seg_row = P.seg_row;
+    h->seg_begin = P.seg_begin;
+    h->hub_seg_ptr = P.hub_seg_ptr;
+    *out = h;
+    return GNNFD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,312 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs.
+
+Bars: CSR structure bit-exact; fp32 aggregation |gpu - oracle| <= 1e-5 * sum|w x| + 1e-6 per element;
+bf16-feature / fp32-accumulate outputs within 1e-2 relative (plus the same absolute terms);
+alpha within 1e-5 relative + 1e-7 and rows summing to 1 within 1e-5.
+"""
+import numpy as np
+import pytest
+
+import graphgen as gg
+import oracle as orc
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+SL, DD, SY = 1, 2, 4
+
+
+@pytest.fixture(scope="module")
+def g():
+    import paper_2104_03058_b200 as lib
+    lib.lib()                     # raises if libgnnfd.so is missing: there is no fallback
+    return lib
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def to_dev_features(w):
+    if w.dtype == "bf16":
+        return torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16)
+    return dev(w.x)
+
+
+def assert_close_f32(got, want, scale, what=""):
+    err = np.abs(got.astype(np.float64) - want)
+    bound = 1e-5 * scale + 1e-6
+    bad = err > bound
+    assert not bad.any(), "%s: %d elements out of tolerance, worst %.3e vs bound %.3e" % (
+        what, bad.sum(), err[bad].max(), bound[bad][np.argmax(err[bad])])
+
+
+def assert_close_bf16(got, want, scale, what=""):
+    err = np.abs(got.astype(np.float64) - want)
+    bound = 1e-2 * np.abs(want) + 1e-5 * scale + 1e-6
+    assert (err <= bound).all(), "%s: worst excess %.3e" % (what, (err - bound).max())
+
+
+def check_csr(g, n, src, dst, flags):
+    csr = g.build_csr(n, dev(src), dev(dst), flags)
+    row_ptr, col, perm = orc.build_csr(n, src, dst, flags)
+    assert csr.nnz == len(col)
+    np.testing.assert_array_equal(csr.row_ptr.cpu().numpy(), row_ptr)
+    np.testing.assert_array_equal(csr.col_idx.cpu().numpy(), col)
+    np.testing.assert_array_equal(csr.perm.cpu().numpy(), perm)
+    deg, dinv, rdeg = orc.degree_norm(row_ptr)
+    assert csr.max_degree == (deg.max() if n else 0)
+    np.testing.assert_array_equal(csr.dinv_sqrt.cpu().numpy(), dinv.astype(np.float32))
+    np.testing.assert_array_equal(csr.rdeg.cpu().numpy(), rdeg.astype(np.float32))
+    rows = np.repeat(np.arange(n), deg)
+    d32 = dinv.astype(np.float32)
+    np.testing.assert_array_equal(csr.edge_weight.cpu().numpy(), d32[col] * d32[rows])
+    check_schedule(g, csr, deg)
+    return csr, (row_ptr, col, perm)
+
+
+def check_schedule(g, csr, deg):
+    order = csr.row_order.cpu().numpy()
+    n = len(deg)
+    assert sorted(order.tolist()) == list(range(n))
+    bounds = [8, 32, 128, g.HUB_DEGREE]
+    bins = np.searchsorted(bounds, deg, side="left")          # first bound >= deg; 4 = hub
+    start = 0
+    for b in range(5):
+        part = order[start:start + csr.bin_count[b]]
+        assert (bins[part] == b).all() and (np.diff(part) > 0).all()
+        start += csr.bin_count[b]
+    assert start == n
+    hubs = order[n - csr.bin_count[4]:]
+    seg_ptr = csr.hub_seg_ptr.cpu().numpy()
+    seg_row = csr.seg_row.cpu().numpy()
+    seg_begin = csr.seg_begin.cpu().numpy()
+    row_ptr = csr.row_ptr.cpu().numpy()
+    assert seg_ptr[0] == 0 and seg_ptr[-1] == csr.n_segments
+    for i, v in enumerate(hubs):
+        want = np.arange(row_ptr[v], row_ptr[v + 1], g.HUB_SEGMENT)
+        np.testing.assert_array_equal(seg_begin[seg_ptr[i]:seg_ptr[i + 1]], want)
+        assert (seg_row[seg_ptr[i]:seg_ptr[i + 1]] == v).all()
+
+
+# ------------------------------------------------------------------ CSR build
+
+@pytest.mark.parametrize("flags", [0, SL, DD, SY, SL | DD, SY | DD | SL])
+@pytest.mark.parametrize("n,e", [(50, 400), (1000, 30_011), (70_000, 9_000)])
+def test_csr_bit_exact_multigraph(g, flags, n, e):
+    src, dst = gg.uniform_graph(n, e, seed=n + flags)
+    check_csr(g, n, src, dst, flags)
+
+
+def test_csr_int64_ids_and_hub_rows(g):
+    n = 3000
+    src, dst = gg.uniform_graph(n, 40_000, seed=3)
+    dst[:9000] = 7                      # one row above the hub threshold, with duplicates
+    dst[9000:12_500] = 11
+    csr, _ = check_csr(g, n, src.astype(np.int64), dst.astype(np.int64), SL)
+    assert csr.bin_count[4] == 2 and csr.n_segments >= 6
+
+
+def test_csr_degenerate_inputs(g):
+    empty = np.zeros(0, np.int32)
+    check_csr(g, 1, empty, empty, 0)
+    check_csr(g, 5, empty, empty, SL)
+    check_csr(g, 1, np.zeros(3, np.int32), np.zeros(3, np.int32), DD)
+    check_csr(g, 2, np.array([0, 1, 1], np.int32), np.array([1, 0, 0], np.int32), SY | DD)
+
+
+def test_csr_rejects_bad_ids_without_fault(g):
+    src = np.array([0, 9, 2], np.int32)
+    dst = np.array([1, 2, -4], np.int32)
+    with pytest.raises(g.GnnfdError) as err:
+        g.build_csr(5, dev(src), dev(dst), 0)
+    assert err.value.status == g.BAD_INDEX
+    # the context is still usable
+    check_csr(g, 5, np.array([0, 4], np.int32), np.array([1, 2], np.int32), 0)
+
+
+def test_workspace_too_small_and_invalid_args(g):
+    src, dst = gg.uniform_graph(100, 1000, seed=1)
+    pb, sb = g.csr_workspace_bytes(100, 1000, 0)
+    small = torch.empty(pb // 2, dtype=torch.uint8, device="cuda")
+    with pytest.raises(g.GnnfdError) as err:
+        g.build_csr(100, dev(src), dev(dst), 0, persistent=small)
+    assert err.value.status == g.WORKSPACE_TOO_SMALL
+    csr = g.build_csr(100, dev(src), dev(dst), 0)
+    x = torch.zeros((100, 8), device="cuda")
+    with pytest.raises(g.GnnfdError) as err:
+        g.aggregate_gcn(csr, x, f=8, chunk_width=0)
+    assert err.value.status == g.INVALID_ARG
+    with pytest.raises(g.GnnfdError):
+        g.csr_workspace_bytes(0, 10, 0)
+    with pytest.raises(g.GnnfdError) as err:
+        g.csr_workspace_bytes(10, 2 ** 31, 0)
+    assert err.value.status == g.TOO_LARGE
+
+
+# ------------------------------------------------------------------ GCN / SAGE
+
+def run_model(g, w, csr, xd, width, out_dtype=None):
+    fn = g.aggregate_gcn if w.model == "gcn" else g.aggregate_sage
+    out = fn(csr, xd, f=w.f, chunk_width=width, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    return out
+
+
+def check_workload(g, w, widths=None, rows=None):
+    csr, (row_ptr, col, _) = check_csr(g, w.n, w.src, w.dst, w.flags)
+    xd = to_dev_features(w)
+    want, scale = orc.aggregate(w.model, row_ptr, col, w.x, w.f, rows=rows, threads=orc.max_threads())
+    for width in widths or w.chunk_widths:
+        got = run_model(g, w, csr, xd, width).cpu().numpy()
+        assert got.shape == (w.n, w.f)
+        if rows is not None:
+            got = got[rows]
+        (assert_close_bf16 if w.dtype == "bf16" else assert_close_f32)(got, want, scale, "%s width %d" % (w.name, width))
+    return csr
+
+
+def test_config1_gcn(g):
+    w = gg.config1()
+    check_workload(g, w, widths=(4, 8, 16, 1, 3, 5, 100))
+
+
+def test_config2_sage(g):
+    w = gg.config2()
+    check_workload(g, w)
+
+
+def test_config4_scaled_gcn_with_hub_rows_and_padding(g):
+    w = gg.scaled("config4", 0.05)
+    w.x[:, w.f:] = np.nan                      # padding columns must never reach a result
+    csr = check_workload(g, w, widths=(32, 64, 128, 602, 7))
+    assert csr.bin_count[4] > 0, "the scaled workload should still contain hub rows"
+
+
+@pytest.mark.parametrize("f", [256, 8, 16, 32, 64])
+def test_config5_scaled_gcn_bf16(g, f):
+    w = gg.scaled("config5_f%d" % f, 1.0 / 64)
+    check_workload(g, w, widths=w.chunk_widths + (4,))
+
+
+def test_bf16_output_and_sage_on_bf16(g):
+    w = gg.scaled("config5_f64", 1.0 / 256)
+    row_ptr, col, _ = orc.build_csr(w.n, w.src, w.dst, w.flags)
+    csr = g.build_csr(w.n, dev(w.src), dev(w.dst), w.flags)
+    xd = to_dev_features(w)
+    for model, fn in (("gcn", g.aggregate_gcn), ("sage", g.aggregate_sage)):
+        want, scale = orc.aggregate(model, row_ptr, col, w.x, w.f)
+        out = fn(csr, xd, f=w.f, chunk_width=16, out_dtype=torch.bfloat16)
+        assert out.dtype == torch.bfloat16
+        got = out.float().cpu().numpy()
+        err = np.abs(got - want)
+        assert (err <= 2.0 ** -8 * np.abs(want) + 1e-2 * np.abs(want) + 1e-5 * scale + 1e-6).all()
+
+
+@pytest.mark.parametrize("model", ["gcn", "sage"])
+def test_unaligned_layouts_take_the_narrow_path(g, model):
+    n, f = 5000, 13
+    src, dst = gg.powerlaw_graph(n, 60_000, 2.1, None, 4)
+    x = gg.features_f32(n, f + 1, dist="normal", p0=0, p1=1, seed=4)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, SL)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    xd = dev(x)
+    view = xd[:, 1:]                            # 4-byte aligned base, odd leading dimension
+    ref = np.ascontiguousarray(x[:, 1:])
+    want, scale = orc.aggregate(model, row_ptr, col, ref, f)
+    fn = g.aggregate_gcn if model == "gcn" else g.aggregate_sage
+    out_buf = torch.full((n, f + 2), -5.0, device="cuda")
+    for width in (13, 4, 8, 1):
+        out = fn(csr, view, f=f, chunk_width=width, out=out_buf[:, 1:f + 1])
+        got = out.cpu().numpy()
+        assert_close_f32(got, want, scale, "%s unaligned width %d" % (model, width))
+        assert (out_buf[:, 0] == -5.0).all() and (out_buf[:, f + 1] == -5.0).all()
+
+
+def test_results_are_bit_identical_from_run_to_run(g):
+    w = gg.scaled("config4", 0.03)
+    csr = g.build_csr(w.n, dev(w.src), dev(w.dst), w.flags)
+    csr2 = g.build_csr(w.n, dev(w.src), dev(w.dst), w.flags)
+    assert torch.equal(csr.col_idx, csr2.col_idx) and torch.equal(csr.perm, csr2.perm)
+    xd = to_dev_features(w)
+    a = g.aggregate_gcn(csr, xd, f=w.f, chunk_width=64)
+    b = g.aggregate_gcn(csr2, xd, f=w.f, chunk_width=64)
+    assert torch.equal(a, b)
+
+
+def test_launch_counter_and_kernel_timing(g):
+    w = gg.config1()
+    before = g.launch_count()
+    csr = g.build_csr(w.n, dev(w.src), dev(w.dst), w.flags)
+    g.kernel_timing_enable(True)
+    try:
+        g.aggregate_gcn(csr, dev(w.x), f=w.f, chunk_width=8)
+        torch.cuda.synchronize()
+        timing = g.kernel_timing_read()
+    finally:
+        g.kernel_timing_enable(False)
+    assert g.launch_count() > before
+    assert "gather_aggregate_gcn" in timing and timing["gather_aggregate_gcn"][1] == 1
+    assert timing["gather_aggregate_gcn"][0] > 0
+
+
+# ------------------------------------------------------------------ GAT
+
+def test_config3_gat_and_edge_softmax(g):
+    w = gg.config3()
+    csr, (row_ptr, col, _) = check_csr(g, w.n, w.src, w.dst, w.flags)
+    zd = dev(w.x)
+    a_src, a_dst = dev(w.a_src), dev(w.a_dst)
+    threads = orc.max_threads()
+    want, scale = orc.aggregate_gat(row_ptr, col, w.x, w.a_src, w.a_dst, w.heads, w.dim, w.negative_slope,
+                                    threads=threads)
+    for width in (8, 64, 16, 4, 24):
+        got = g.aggregate_gat(csr, zd, a_src, a_dst, w.heads, w.dim, w.negative_slope, chunk_width=width)
+        assert_close_f32(got.cpu().numpy(), want, scale, "gat width %d" % width)
+    # scores and the materialised softmax
+    s_src, s_dst = g.gat_scores(zd, a_src, a_dst, w.heads, w.dim)
+    o_src, o_dst = orc.gat_scores(w.x, w.a_src, w.a_dst, w.heads, w.dim)
+    zz = np.abs(w.x.astype(np.float64)).reshape(w.n, w.heads, w.dim)
+    s_scale = np.einsum("nhd,hd->nh", zz, np.abs(w.a_src.astype(np.float64)))
+    assert_close_f32(s_src.cpu().numpy(), o_src, s_scale, "s_src")
+    alpha = g.edge_softmax(csr, s_src, s_dst, w.negative_slope).cpu().numpy()
+    want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), w.negative_slope)
+    assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
+    sums = np.add.reduceat(alpha.astype(np.float64), row_ptr[:-1], axis=0)
+    assert np.abs(sums - 1.0).max() <= 1e-5
+
+
+@pytest.mark.parametrize("heads,dim", [(3, 5), (1, 7), (4, 4), (2, 64)])
+def test_gat_general_shapes_with_hub_rows(g, heads, dim):
+    n = 6000
+    src, dst = gg.powerlaw_graph(n, 90_000, 2.1, None, heads)
+    dst[:5000] = 17                     # guarantees a row above the hub threshold
+    f = heads * dim
+    z = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=heads)
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=heads, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=heads, stream=6)
+    csr, (row_ptr, col, _) = check_csr(g, n, src, dst, SL)
+    assert csr.bin_count[4] > 0
+    want, scale = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2, threads=orc.max_threads())
+    for width in sorted({f, dim, 4, 3}):
+        got = g.aggregate_gat(csr, dev(z), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
+        assert_close_f32(got.cpu().numpy(), want, scale, "gat %dx%d width %d" % (heads, dim, width))
+    s_src, s_dst = g.gat_scores(dev(z), dev(a_src), dev(a_dst), heads, dim)
+    alpha = g.edge_softmax(csr, s_src, s_dst, 0.2).cpu().numpy()
+    want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), 0.2)
+    assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
+
+
+def test_gat_bf16_features(g):
+    n, heads, dim = 4000, 4, 8
+    src, dst = gg.powerlaw_graph(n, 50_000, 2.1, None, 9)
+    bits = gg.to_bf16_bits(gg.features_f32(n, heads * dim, dist="normal", p0=0, p1=1, seed=9))
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.1, seed=9, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.1, seed=9, stream=6)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, SL)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    zd = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    want, scale = orc.aggregate_gat(row_ptr, col, bits, a_src, a_dst, heads, dim, 0.2)
+    for width in (8, 32, 2):
+        got = g.aggregate_gat(csr, zd, dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
+        assert_close_bf16(got.cpu().numpy(), want, scale, "gat bf16 width %d" % width)
