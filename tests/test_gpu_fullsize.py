@@ -1,0 +1,63 @@
+"""Full-size parity: config 4 exactly as bench.py launches it (232,965 vertices, ~115M edges,
+F = 602 in rows of 608, chunk width 64).  The CSR is compared bit for bit with the oracle's; the
+aggregation on sampled rows (every degree class and the hub rows included) element by element, and on
+all rows through closed forms that hold at any size."""
+import numpy as np
+import pytest
+
+import graphgen as gg
+import oracle as orc
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def big():
+    import paper_2104_03058_b200 as g
+    w = gg.config4()
+    row_ptr, col, perm = orc.build_csr(w.n, w.src, w.dst, w.flags)
+    csr = g.build_csr(w.n, torch.from_numpy(w.src).cuda(), torch.from_numpy(w.dst).cuda(), w.flags)
+    return g, w, csr, (row_ptr, col, perm)
+
+
+def test_config4_csr_bit_exact(big):
+    g, w, csr, (row_ptr, col, perm) = big
+    assert csr.nnz == len(col) and abs(csr.nnz - w.n - 114_615_892) < 0.02 * 114_615_892
+    assert torch.equal(csr.row_ptr.cpu(), torch.from_numpy(row_ptr))
+    assert torch.equal(csr.col_idx.cpu(), torch.from_numpy(col))
+    assert torch.equal(csr.perm.cpu(), torch.from_numpy(perm))
+    assert csr.max_degree == int(np.diff(row_ptr).max()) and csr.bin_count[4] > 1000
+
+
+def test_config4_gcn_sampled_rows_in_the_bench_configuration(big):
+    g, w, csr, (row_ptr, col, _) = big
+    deg = np.diff(row_ptr)
+    rng = np.random.default_rng(4)
+    rows = np.concatenate([rng.choice(w.n, 192, replace=False), np.argsort(deg)[-16:], np.argsort(deg)[:16]])
+    rows = np.unique(rows).astype(np.int64)
+    want, scale = orc.aggregate("gcn", row_ptr, col, w.x, w.f, rows=rows, threads=orc.max_threads())
+    xd = torch.from_numpy(w.x).cuda()
+    out = torch.full((w.n, w.ld), float("nan"), device="cuda")
+    for width in (64, 128, 602):
+        out.fill_(float("nan"))
+        g.aggregate_gcn(csr, xd, f=w.f, chunk_width=width, out=out[:, :w.f])
+        torch.cuda.synchronize()
+        got = out[torch.from_numpy(rows).cuda()][:, :w.f].cpu().numpy()
+        err = np.abs(got - want)
+        assert (err <= 1e-5 * scale + 1e-6).all(), "width %d: worst %.3e" % (width, (err - 1e-5 * scale).max())
+        assert bool(torch.isnan(out[:, w.f:]).all()) and not bool(torch.isnan(out[:, :w.f]).any())
+
+
+def test_config4_closed_forms_on_every_row(big):
+    g, w, csr, (row_ptr, _, _) = big
+    deg = np.diff(row_ptr).astype(np.float64)
+    # x[u, :] = sqrt(deg u)  =>  GCN out[v, :] = sum_u deg_u^-1/2 deg_v^-1/2 sqrt(deg_u) = sqrt(deg v)
+    f = 8
+    x = torch.from_numpy(np.repeat(np.sqrt(deg)[:, None], f, axis=1).astype(np.float32)).cuda()
+    got = g.aggregate_gcn(csr, x, f=f, chunk_width=4).cpu().numpy()
+    np.testing.assert_allclose(got, np.sqrt(deg)[:, None] * np.ones((1, f)), rtol=2e-5)
+    # the mean of a constant is the constant
+    c = torch.full((w.n, f), 3.25, device="cuda")
+    got = g.aggregate_sage(csr, c, f=f, chunk_width=8).cpu().numpy()
+    np.testing.assert_allclose(got, 3.25, rtol=2e-5)
