@@ -52,7 +52,8 @@ typedef enum {
     GNNFD_TOO_LARGE = -3,           /* n, e or the resulting nnz does not fit the int32 structure */
     GNNFD_WORKSPACE_TOO_SMALL = -4, /* a caller-provided buffer is smaller than the size query says */
     GNNFD_UNSUPPORTED = -5,         /* unknown dtype / itype enum */
-    GNNFD_CUDA_ERROR = -6           /* a CUDA runtime call failed; see gnnfd_last_cuda_error() */
+    GNNFD_CUDA_ERROR = -6,          /* a CUDA runtime call failed; see gnnfd_last_cuda_error() */
+    GNNFD_STATIC_SCRATCH_EXCEEDED = -7 /* the built-in workspace of a *_static entry point is too small for this call */
 } gnnfd_status_t;
 
 /* ------------------------------------------------------------------ graph set-up
@@ -115,7 +116,8 @@ void gnnfd_csr_destroy(gnnfd_csr_t* csr);
  * chunk_width (>= 1) is the width of one decomposition layer: P = ceil(f / chunk_width) chunks, the
  * last one narrower; chunk_width >= f means no decomposition.  Chunks are swept one after the other
  * over all rows, so the gathered working set of a sweep is n * chunk_width elements.  The result
- * does not depend on chunk_width beyond fp32 rounding of identical sums (it is in fact bit-identical).
+ * does not depend on chunk_width beyond fp32 rounding (the order of the additions inside a row
+ * depends on how many lanes a chunk occupies).
  *
  * d_x: [n, ldx] of xdt.  d_out: [n, ldo] of odt (must not alias d_x).  d_scratch: per-call buffer
  * of gnnfd_aggregate_workspace_bytes(csr, f) bytes (holds the per-segment partial sums of hub rows;
@@ -131,6 +133,32 @@ int gnnfd_aggregate_gcn(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gn
 int gnnfd_aggregate_sage(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt,
                          void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
                          void* d_scratch, size_t scratch_bytes, void* stream);
+
+/* GCN aggregation without a caller workspace and without any allocation.  (The paper has no
+ * counterpart to this entry point; it exists for the library's users.)
+ *
+ * Who needs it: a host that gave the whole device to its own memory pool at start-up, or that calls
+ * from a loop where cudaMalloc's device-wide synchronisation is not acceptable, and that has no spare
+ * buffer to hand over.  Such a caller cannot obtain the hub-row workspace gnnfd_aggregate_gcn asks
+ * for.  Here that workspace is a fixed array of GNNFD_STATIC_SCRATCH_BYTES inside the library image;
+ * every device that loads the library carries it until the process exits.  The call itself performs
+ * no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Same arguments and same results (bit for bit) as gnnfd_aggregate_gcn, minus the scratch pair.
+ * Limits and rules:
+ *   - returns GNNFD_STATIC_SCRATCH_EXCEEDED when gnnfd_aggregate_workspace_bytes(csr, f) is larger
+ *     than GNNFD_STATIC_SCRATCH_BYTES (hub segments x f rounded up to 4, x 4 bytes); nothing is launched;
+ *   - the first call on each device looks up the array's device address (one runtime query, with that
+ *     device current); make that first call outside any stream capture;
+ *   - all calls on a device share the one array and it keeps whatever the previous call left.  The
+ *     kernels overwrite every element before reading it, so nothing needs clearing, but two calls
+ *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on it:
+ *     serialise them, or use gnnfd_aggregate_gcn with separate buffers. */
+#define GNNFD_STATIC_SCRATCH_BYTES (32u << 20)
+
+int gnnfd_aggregate_gcn_static(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt,
+                               void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
+                               void* stream);
 
 /* ------------------------------------------------------------------ GAT
  *

@@ -17,6 +17,8 @@ F32, BF16 = 0, 1
 I32, I64 = 0, 1
 CSR_ADD_SELF_LOOPS, CSR_DEDUP, CSR_SYMMETRIZE = 1, 2, 4
 OK, INVALID_ARG, BAD_INDEX, TOO_LARGE, WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA_ERROR = 0, -1, -2, -3, -4, -5, -6
+STATIC_SCRATCH_EXCEEDED = -7
+STATIC_SCRATCH_BYTES = 32 << 20
 HUB_DEGREE, HUB_SEGMENT = 2048, 1024
 
 _lib = None
@@ -52,6 +54,7 @@ def lib() -> ctypes.CDLL:
         agg = [vp, vp, i64, i32, vp, i64, i32, i32, i32, vp, sz, vp]
         L.gnnfd_aggregate_gcn.argtypes = agg
         L.gnnfd_aggregate_sage.argtypes = agg
+        L.gnnfd_aggregate_gcn_static.argtypes = [vp, vp, i64, i32, vp, i64, i32, i32, i32, vp]
         L.gnnfd_gat_scores.argtypes = [i64, vp, i64, i32, vp, vp, i32, i32, vp, vp, vp]
         L.gnnfd_gat_workspace_bytes.argtypes = [vp, i32, i32, pp(sz)]
         L.gnnfd_aggregate_gat.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32, vp, sz, vp]
@@ -218,6 +221,23 @@ def aggregate_sage(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width:
                    out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None) -> torch.Tensor:
     return _aggregate(lib().gnnfd_aggregate_sage, "gnnfd_aggregate_sage", csr, x, f, chunk_width, out, out_dtype,
                       scratch, stream)
+
+
+def aggregate_gcn_static(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width: int | None = None,
+                         out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """gnnfd_aggregate_gcn_static: GCN aggregation whose hub-row workspace is the library's built-in
+    array, for callers that can neither allocate device memory nor spare a buffer.  ``out`` should be
+    passed by such callers (when it is None this wrapper allocates it with torch, which the C entry
+    point itself never does).  Raises GnnfdError(STATIC_SCRATCH_EXCEEDED) beyond the built-in size."""
+    f = x.shape[1] if f is None else f
+    chunk_width = f if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((csr.n, f), dtype=torch.float32, device=x.device)
+    xp, ldx = _matrix(x, f, "x")
+    op, ldo = _matrix(out, f, "out")
+    _check(lib().gnnfd_aggregate_gcn_static(csr.handle, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f,
+                                            chunk_width, _stream_ptr(stream)), "gnnfd_aggregate_gcn_static")
+    return out
 
 
 def gat_scores(z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.Tensor, heads: int, dim: int, stream=None):

@@ -153,6 +153,7 @@ const char* gnnfd_status_string(int status)
         case GNNFD_WORKSPACE_TOO_SMALL: return "workspace buffer too small";
         case GNNFD_UNSUPPORTED: return "unsupported dtype or index type";
         case GNNFD_CUDA_ERROR: return "CUDA runtime error";
+        case GNNFD_STATIC_SCRATCH_EXCEEDED: return "built-in workspace too small for this call";
         default: return "unknown status";
     }
 }
