@@ -105,21 +105,32 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     for (int i = 0; i < VECN; ++i) acc[i] = 0.f;
     const T* xj = static_cast<const T*>(a.x) + j;
 
-    for (int32_t k = b + g; k < e; k += EP * kUnroll) {
-        int32_t u[kUnroll];
-        float w[kUnroll];
+    // Software pipeline: the indices (and weights) of step i+1 are requested right after the feature
+    // loads of step i are issued, so the index stream from HBM overlaps the gathers from L2.
+    int32_t u[kUnroll];
+    float w[kUnroll];
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            const int32_t kk = k + t * EP;
-            const bool ok = kk < e;
-            u[t] = ok ? __ldcs(a.col_idx + kk) : -1;
-            if (WEIGHTED) w[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
-        }
+    for (int t = 0; t < kUnroll; ++t) {
+        const int32_t kk = b + g + t * EP;
+        const bool ok = kk < e;
+        u[t] = ok ? __ldcs(a.col_idx + kk) : -1;
+        if (WEIGHTED) w[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
+    }
+    for (int32_t k = b + g; k < e; k += EP * kUnroll) {
         Vec<T, VECN> v[kUnroll];
 #pragma unroll
         for (int t = 0; t < kUnroll; ++t) {
             if (u[t] >= 0 && col_ok) v[t].load(xj + (int64_t)u[t] * a.ldx);
             else v[t].zero();
+        }
+        int32_t un[kUnroll];
+        float wn[kUnroll];
+#pragma unroll
+        for (int t = 0; t < kUnroll; ++t) {
+            const int32_t kk = k + (kUnroll + t) * EP;
+            const bool ok = kk < e;
+            un[t] = ok ? __ldcs(a.col_idx + kk) : -1;
+            if (WEIGHTED) wn[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
         }
 #pragma unroll
         for (int t = 0; t < kUnroll; ++t) {
@@ -128,6 +139,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
                 if (WEIGHTED) acc[i] = fmaf(w[t], v[t].get(i), acc[i]);
                 else acc[i] += v[t].get(i);
             }
+            u[t] = un[t];
+            if (WEIGHTED) w[t] = wn[t];
         }
     }
 

@@ -12,8 +12,8 @@ namespace gnnfd {
 using u64 = unsigned long long;
 
 constexpr int kThreads = 256;
-constexpr int kRadixBits = 8;
-constexpr int kRadix = 1 << kRadixBits;
+constexpr int kMaxDigitBits = 9;
+constexpr int kRadix = 1 << kMaxDigitBits;           // histogram bins (a pass may use fewer)
 constexpr int kSortItems = 16;                       // keys per thread
 constexpr int kSortTile = kThreads * kSortItems;     // keys per block
 constexpr int kSortWarps = kThreads / 32;
@@ -28,15 +28,15 @@ static inline unsigned blocks_for(size_t count, int per_block)
 // ------------------------------------------------------------------ keys
 
 // Candidate i < e: input edge i.  e <= i < 2e (symmetrise): reverse of edge i - e.  Then one
-// self-loop per vertex (value -1).  Dropped candidates get the key 1 << (2*bits), above every
-// valid key, so the sort moves them behind the kept ones.
+// self-loop per vertex (value -1).  key = (dst << src_bits) | src; dropped candidates get the
+// destination n, above every valid key, so the sort moves them behind the kept ones.
 template <typename IdT>
 __global__ void __launch_bounds__(kThreads)
 make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, int64_t e, int64_t m, uint32_t flags,
-          int bits, u64* __restrict__ keys, int32_t* __restrict__ vals, BuildCounts* __restrict__ counts)
+          int src_bits, u64* __restrict__ keys, int32_t* __restrict__ vals, BuildCounts* __restrict__ counts)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    const u64 invalid = 1ull << (2 * bits);
+    const u64 invalid = (u64)n << src_bits;
     const int64_t n_rev = (flags & GNNFD_CSR_SYMMETRIZE) ? e : 0;
     bool keep = false, bad = false;
     if (i < m) {
@@ -53,66 +53,109 @@ make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, i
             s = d = i - e - n_rev; val = -1;
             keep = true;
         }
-        keys[i] = keep ? (((u64)d << bits) | (u64)s) : invalid;
-        vals[i] = val;
+        __stcs(keys + i, keep ? (((u64)d << src_bits) | (u64)s) : invalid);
+        __stcs(vals + i, val);
     }
-    const unsigned kept = __ballot_sync(0xffffffffu, keep);
-    const unsigned bads = __ballot_sync(0xffffffffu, bad);
-    if ((threadIdx.x & 31) == 0) {
-        if (kept) atomicAdd(&counts->n_valid, __popc(kept));
-        if (bads) atomicAdd(&counts->bad_index, __popc(bads));
+    const int kept = __syncthreads_count(keep);
+    const int bads = __syncthreads_count(bad);
+    if (threadIdx.x == 0) {
+        if (kept) atomicAdd(&counts->n_valid, kept);
+        if (bads) atomicAdd(&counts->bad_index, bads);
     }
 }
 
-// ------------------------------------------------------------------ radix sort (one 8-bit digit per pass)
+// ------------------------------------------------------------------ radix sort (one digit of up to 9 bits per pass)
 
 __global__ void __launch_bounds__(kThreads)
-radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int64_t n_tiles, int32_t* __restrict__ hist)
+radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int mask, int64_t n_tiles, int32_t* __restrict__ hist)
 {
     __shared__ int32_t h[kRadix];
     h[threadIdx.x] = 0;
+    h[threadIdx.x + kThreads] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
 #pragma unroll
     for (int i = 0; i < kSortItems; ++i) {
         const int64_t idx = base + i * kThreads + threadIdx.x;
-        if (idx < m) atomicAdd(&h[(int)((keys[idx] >> shift) & (kRadix - 1))], 1);
+        if (idx < m) atomicAdd(&h[(int)(keys[idx] >> shift) & mask], 1);
     }
     __syncthreads();
     hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
+    hist[(int64_t)(threadIdx.x + kThreads) * n_tiles + blockIdx.x] = h[threadIdx.x + kThreads];
 }
 
-// Stable scatter.  A warp owns 512 consecutive keys of the tile and walks them 32 at a time; keys
-// with equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp
-// running count, across warps by a prefix over the per-warp counts, across tiles by the scanned
-// histogram.
-__global__ void __launch_bounds__(kThreads)
+struct ScatterSmem {
+    u64 keys[kSortTile];
+    int32_t vals[kSortTile];
+    int32_t warp_count[kSortWarps][kRadix];
+    int32_t digit_base[kRadix];     // first slot of each digit inside the sorted tile
+    int32_t to_global[kRadix];      // global position of tile slot i holding digit d: to_global[d] + i
+    int32_t scan[kSortWarps];
+};
+
+// exclusive scan of one value per thread over the block; *total receives the block sum
+__device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int32_t* smem)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    int32_t off = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+        const int32_t s = smem[w];
+        if (w < warp) off += s;
+        all += s;
+    }
+    *total = all;
+    return off + inc - v;
+}
+
+// Stable scatter of one tile.  A warp owns 512 consecutive keys and walks them 32 at a time: keys with
+// equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp running
+// count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
+// digit in shared memory and written out run by run, so that consecutive threads store to
+// consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
+__global__ void __launch_bounds__(kThreads, 3)
 radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_in, u64* __restrict__ keys_out,
-              int32_t* __restrict__ vals_out, int64_t m, int shift, int64_t n_tiles,
+              int32_t* __restrict__ vals_out, int64_t m, int shift, int mask, int64_t n_tiles,
               const int32_t* __restrict__ tile_offset)
 {
-    __shared__ int32_t warp_count[kSortWarps][kRadix];
-    __shared__ int32_t global_base[kRadix];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ScatterSmem& sm = *reinterpret_cast<ScatterSmem*>(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-    for (int w = 0; w < kSortWarps; ++w) warp_count[w][threadIdx.x] = 0;
+    for (int w = 0; w < kSortWarps; ++w) {
+        sm.warp_count[w][threadIdx.x] = 0;
+        sm.warp_count[w][threadIdx.x + kThreads] = 0;
+    }
     __syncthreads();
 
-    const int64_t warp_base = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * kWarpItems;
+    const int64_t tile_base = (int64_t)blockIdx.x * kSortTile;
+    const int64_t warp_base = tile_base + (int64_t)warp * kWarpItems;
     u64 key[kSortItems];
-    int32_t rank[kSortItems];
 #pragma unroll
     for (int r = 0; r < kSortItems; ++r) {
         const int64_t idx = warp_base + r * 32 + lane;
-        const bool valid = idx < m;
-        key[r] = valid ? keys_in[idx] : 0ull;
-        const int digit = valid ? (int)((key[r] >> shift) & (kRadix - 1)) : kRadix;
+        key[r] = idx < m ? __ldcs(keys_in + idx) : 0ull;
+    }
+    int32_t rank[kSortItems];
+#pragma unroll
+    for (int r = 0; r < kSortItems; ++r) {
+        const bool valid = warp_base + r * 32 + lane < m;
+        const int digit = valid ? ((int)(key[r] >> shift) & mask) : kRadix;
         const unsigned peers = __match_any_sync(0xffffffffu, digit);
         const int leader = __ffs(peers) - 1;
         int32_t before = 0;
         if (lane == leader && valid) {
-            before = warp_count[warp][digit];
-            warp_count[warp][digit] = before + __popc(peers);
+            before = sm.warp_count[warp][digit];
+            sm.warp_count[warp][digit] = before + __popc(peers);
         }
         before = __shfl_sync(0xffffffffu, before, leader);
         rank[r] = before + __popc(peers & ((1u << lane) - 1u));
@@ -120,25 +163,46 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
     }
     __syncthreads();
     {
-        int32_t run = 0;
+        // per-warp counts -> exclusive prefix over warps; thread t owns digits t and t + 256
+        int32_t tot[2];
 #pragma unroll
-        for (int w = 0; w < kSortWarps; ++w) {
-            const int32_t c = warp_count[w][threadIdx.x];
-            warp_count[w][threadIdx.x] = run;
-            run += c;
+        for (int half = 0; half < 2; ++half) {
+            const int d = threadIdx.x + half * kThreads;
+            int32_t run = 0;
+#pragma unroll
+            for (int w = 0; w < kSortWarps; ++w) {
+                const int32_t c = sm.warp_count[w][d];
+                sm.warp_count[w][d] = run;
+                run += c;
+            }
+            tot[half] = run;
         }
-        global_base[threadIdx.x] = tile_offset[(int64_t)threadIdx.x * n_tiles + blockIdx.x];
+        int32_t low_total, high_total;
+        const int32_t base0 = block_scan_256(tot[0], &low_total, sm.scan);
+        const int32_t base1 = block_scan_256(tot[1], &high_total, sm.scan) + low_total;
+        sm.digit_base[threadIdx.x] = base0;
+        sm.digit_base[threadIdx.x + kThreads] = base1;
+        sm.to_global[threadIdx.x] = tile_offset[(int64_t)threadIdx.x * n_tiles + blockIdx.x] - base0;
+        sm.to_global[threadIdx.x + kThreads] =
+            tile_offset[(int64_t)(threadIdx.x + kThreads) * n_tiles + blockIdx.x] - base1;
     }
     __syncthreads();
 #pragma unroll
     for (int r = 0; r < kSortItems; ++r) {
-        const int64_t idx = warp_base + r * 32 + lane;
-        if (idx < m) {
-            const int digit = (int)((key[r] >> shift) & (kRadix - 1));
-            const int64_t pos = (int64_t)global_base[digit] + warp_count[warp][digit] + rank[r];
-            keys_out[pos] = key[r];
-            vals_out[pos] = vals_in[idx];
+        if (warp_base + r * 32 + lane < m) {
+            const int digit = (int)(key[r] >> shift) & mask;
+            const int slot = sm.digit_base[digit] + sm.warp_count[warp][digit] + rank[r];
+            sm.keys[slot] = key[r];
+            sm.vals[slot] = __ldcs(vals_in + warp_base + r * 32 + lane);
         }
+    }
+    __syncthreads();
+    const int count = (int)min((int64_t)kSortTile, m - tile_base);
+    for (int i = threadIdx.x; i < count; i += kThreads) {
+        const u64 k = sm.keys[i];
+        const int64_t pos = (int64_t)sm.to_global[(int)(k >> shift) & mask] + i;
+        keys_out[pos] = k;
+        vals_out[pos] = sm.vals[i];
     }
 }
 
@@ -168,23 +232,18 @@ compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, c
     if (i == m - 1) counts->nnz = pos[i] + flag[i];
 }
 
+// row_ptr[v] = number of kept keys with dst < v (binary search in the sorted keys).  Without
+// duplicate removal every kept candidate is an entry, which thread 0 records.
 __global__ void __launch_bounds__(kThreads)
-copy_perm(const int32_t* __restrict__ vals, int64_t m, int32_t* __restrict__ perm, BuildCounts* __restrict__ counts)
-{
-    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (i == 0) counts->nnz = counts->n_valid;
-    if (i < m && i < counts->n_valid) perm[i] = vals[i];
-}
-
-// row_ptr[v] = number of kept keys with dst < v (binary search in the sorted keys)
-__global__ void __launch_bounds__(kThreads)
-row_pointers(const u64* __restrict__ keys, const BuildCounts* __restrict__ counts, int64_t n, int bits,
+row_pointers(const u64* __restrict__ keys, BuildCounts* __restrict__ counts, int64_t n, int src_bits, int dedup,
              int32_t* __restrict__ row_ptr)
 {
     const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const int32_t nnz = dedup ? counts->nnz : counts->n_valid;
+    if (v == 0 && !dedup) counts->nnz = nnz;
     if (v > n) return;
-    const u64 target = (u64)v << bits;
-    int32_t lo = 0, hi = counts->nnz;
+    const u64 target = (u64)v << src_bits;
+    int32_t lo = 0, hi = nnz;
     while (lo < hi) {
         const int32_t mid = lo + ((hi - lo) >> 1);
         if (keys[mid] < target) lo = mid + 1; else hi = mid;
@@ -217,18 +276,20 @@ degrees_and_bins(const int32_t* __restrict__ row_ptr, int64_t n, float* __restri
     if ((threadIdx.x & 31) == 0 && deg > 0) atomicMax(&counts->max_degree, deg);
 }
 
-// col_idx and the GCN weight of every slot, from the sorted keys
+// col_idx, the GCN weight and (unless the duplicate removal already wrote it) perm of every slot
 __global__ void __launch_bounds__(kThreads)
-columns_and_weights(const u64* __restrict__ keys, const BuildCounts* __restrict__ counts, int bits,
-                    const float* __restrict__ dinv, int32_t* __restrict__ col_idx, float* __restrict__ edge_w, int64_t m)
+finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const BuildCounts* __restrict__ counts,
+                 int src_bits, const float* __restrict__ dinv, int32_t* __restrict__ col_idx,
+                 float* __restrict__ edge_w, int32_t* __restrict__ perm, int64_t m)
 {
     const int64_t k = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (k >= m || k >= counts->nnz) return;
-    const u64 key = keys[k];
-    const int32_t s = (int32_t)(key & ((1ull << bits) - 1ull));
-    const int32_t d = (int32_t)(key >> bits);
-    col_idx[k] = s;
-    edge_w[k] = dinv[s] * dinv[d];
+    const u64 key = __ldcs(keys + k);
+    const int32_t s = (int32_t)(key & ((1ull << src_bits) - 1ull));
+    const int32_t d = (int32_t)(key >> src_bits);
+    __stcs(col_idx + k, s);
+    __stcs(edge_w + k, __ldg(dinv + s) * __ldg(dinv + d));
+    if (vals) __stcs(perm + k, __ldcs(vals + k));
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -290,7 +351,7 @@ struct BuildLayout {
     int64_t n_tiles;       // sort tiles
     int64_t hub_cap;       // upper bound on hub rows
     int64_t seg_cap;       // upper bound on hub segments
-    int bits, key_bits, passes;
+    int src_bits, key_bits, passes, digit_bits;
 };
 
 static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
@@ -310,9 +371,12 @@ static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
     L->seg_cap = m / kHubSegment + L->hub_cap + 1;
     int bits = 1;
     while ((int64_t(1) << bits) < n) ++bits;
-    L->bits = bits;
-    L->key_bits = 2 * bits + 1;
-    L->passes = (L->key_bits + kRadixBits - 1) / kRadixBits;
+    int dst_bits = 1;
+    while ((int64_t(1) << dst_bits) < n + 1) ++dst_bits;      // destination n marks dropped candidates
+    L->src_bits = bits;
+    L->key_bits = bits + dst_bits;
+    L->passes = (L->key_bits + kMaxDigitBits - 1) / kMaxDigitBits;
+    L->digit_bits = (L->key_bits + L->passes - 1) / L->passes;
     return GNNFD_OK;
 }
 
@@ -422,27 +486,31 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
     int32_t* vals = S.vals_a;
     int32_t* vals_alt = S.vals_b;
 
+    const bool dedup = (flags & GNNFD_CSR_DEDUP) != 0;
     if (m > 0) {
         if (itype == GNNFD_I32)
             GNNFD_LAUNCH("make_keys", s, make_keys<int32_t>, blocks_for(m, kThreads), kThreads, 0,
-                         static_cast<const int32_t*>(d_src), static_cast<const int32_t*>(d_dst), n, e, m, flags, L.bits,
+                         static_cast<const int32_t*>(d_src), static_cast<const int32_t*>(d_dst), n, e, m, flags, L.src_bits,
                          keys, vals, P.counts);
         else
             GNNFD_LAUNCH("make_keys", s, make_keys<long long>, blocks_for(m, kThreads), kThreads, 0,
                          static_cast<const long long*>(d_src), static_cast<const long long*>(d_dst), n, e, m, flags,
-                         L.bits, keys, vals, P.counts);
+                         L.src_bits, keys, vals, P.counts);
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)sizeof(ScatterSmem)));
+        const int mask = (1 << L.digit_bits) - 1;
         for (int pass = 0; pass < L.passes; ++pass) {
-            const int shift = pass * kRadixBits;
-            GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.n_tiles, kThreads, 0, keys, m, shift,
+            const int shift = pass * L.digit_bits;
+            GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.n_tiles, kThreads, 0, keys, m, shift, mask,
                          L.n_tiles, S.hist);
             rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.n_tiles, S.scan_temp, s);
             if (rc) return rc;
-            GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.n_tiles, kThreads, 0, keys, vals, keys_alt,
-                         vals_alt, m, shift, L.n_tiles, S.hist);
+            GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.n_tiles, kThreads, sizeof(ScatterSmem), keys, vals,
+                         keys_alt, vals_alt, m, shift, mask, L.n_tiles, S.hist);
             u64* tk = keys; keys = keys_alt; keys_alt = tk;
             int32_t* tv = vals; vals = vals_alt; vals_alt = tv;
         }
-        if (flags & GNNFD_CSR_DEDUP) {
+        if (dedup) {
             GNNFD_LAUNCH("flag_first_of_run", s, flag_first_of_run, blocks_for(m, kThreads), kThreads, 0, keys, m,
                          P.counts, S.flags);
             int32_t* pos = vals_alt;   // free after the last pass
@@ -451,17 +519,16 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
             GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys, vals, S.flags,
                          pos, m, keys_alt, P.perm, P.counts);
             keys = keys_alt;
-        } else {
-            GNNFD_LAUNCH("copy_perm", s, copy_perm, blocks_for(m, kThreads), kThreads, 0, vals, m, P.perm, P.counts);
         }
     }
     GNNFD_LAUNCH("row_pointers", s, row_pointers, blocks_for((size_t)n + 1, kThreads), kThreads, 0, keys, P.counts, n,
-                 L.bits, P.row_ptr);
+                 L.src_bits, dedup ? 1 : 0, P.row_ptr);
     GNNFD_LAUNCH("degrees_and_bins", s, degrees_and_bins, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
                  P.dinv, P.rdeg, S.flags, P.counts);
     if (m > 0)
-        GNNFD_LAUNCH("columns_and_weights", s, columns_and_weights, blocks_for(m, kThreads), kThreads, 0, keys, P.counts,
-                     L.bits, P.dinv, P.col_idx, P.edge_w, m);
+        GNNFD_LAUNCH("finalize_entries", s, finalize_entries, blocks_for(m, kThreads), kThreads, 0, keys,
+                     dedup ? (const int32_t*)nullptr : (const int32_t*)vals, P.counts, L.src_bits, P.dinv, P.col_idx,
+                     P.edge_w, P.perm, m);
     rc = exclusive_scan_i32(S.flags, S.flags, (size_t)kNumBins * (size_t)n, S.scan_temp, s);
     if (rc) return rc;
     GNNFD_LAUNCH("place_rows", s, place_rows, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, S.flags, n,
