@@ -95,9 +95,11 @@ int gnnfd_csr_info(const gnnfd_csr_t* csr, int64_t* n, int64_t* nnz, const int32
                    const float** d_rdeg, const float** d_edge_weight, int32_t* max_degree);
 
 /* The launch schedule.  bin_count[5]: rows with degree <= 8, <= 32, <= 128, <= GNNFD_HUB_DEGREE, and
- * hub rows.  d_row_order[n]: row ids grouped by bin (ascending id inside a bin).  Hub segments:
- * d_seg_row[n_segments], d_seg_begin[n_segments] (first CSR slot of the segment);
- * d_hub_seg_ptr[n_hub+1] indexes the segments of the i-th hub row (i-th row of the last bin). */
+ * hub rows.  d_row_order[n]: row ids sorted by degree class, ascending id inside a class; a class is
+ * the exact degree up to 8, then a quarter octave of (degree - 1) up to GNNFD_HUB_DEGREE, then one
+ * class for all hub rows, so every bin is a contiguous range and neighbouring rows have near-equal
+ * lengths.  Hub segments: d_seg_row[n_segments], d_seg_begin[n_segments] (first CSR slot of the
+ * segment); d_hub_seg_ptr[n_hub+1] indexes the segments of the i-th hub row (i-th row of the last bin). */
 int gnnfd_csr_schedule(const gnnfd_csr_t* csr, int64_t bin_count[5], const int32_t** d_row_order,
                        int64_t* n_segments, const int32_t** d_seg_row, const int32_t** d_seg_begin,
                        const int32_t** d_hub_seg_ptr);

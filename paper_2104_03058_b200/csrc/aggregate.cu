@@ -6,8 +6,8 @@
 // chunk-major), so at any time the blocks in flight gather from one chunk's n x chunk_width slice of
 // x, which is what keeps the gathered working set small enough for L2.  Inside a sweep the rows come
 // grouped by degree class.  A row is owned by S = LPR * EP lanes: LPR lanes cover the chunk's columns
-// with one 16-byte vector each, and EP groups of LPR lanes walk interleaved edges of the row, each
-// keeping U loads in flight.  The EP partial sums are combined by a fixed shuffle tree, hub rows
+// with one or two 16-byte vectors each, and EP groups of LPR lanes walk interleaved entries of the
+// row, each keeping 8 loads in flight.  The EP partial sums are combined by a fixed shuffle tree, hub rows
 // (degree > GNNFD_HUB_DEGREE) by per-segment partial sums that a second kernel adds in ascending
 // segment order: no atomics, bit-identical from run to run.
 #include <cuda_bf16.h>
@@ -72,20 +72,41 @@ __device__ __forceinline__ void store_elem(void* out, int out_bf16, int64_t idx,
     else __stcs(static_cast<float*>(out) + idx, val);
 }
 
-// One row (or hub segment) per S = LPR * EP lanes.
-template <typename T, int VECN, int LPR, bool WEIGHTED, int EP>
+constexpr int kLoads = 8;      // 16-byte feature loads kept in flight per lane
+
+// One row (or hub segment) per S = LPR * EP lanes.  The S lanes fetch the row's indices and weights
+// S at a time with one coalesced load each (R rounds per batch) and hand them to one another by
+// shuffle: in step s of a batch, group g works on entry r*S + t*EP + g (r = s / LPR, t = s % LPR),
+// which lane t*EP + g of the segment holds in its r-th register.  A lane covers VPL vectors of the
+// chunk (columns c + q*LPR, q < VPL, in vector units) so that the index traffic, the address
+// arithmetic and the shuffles are paid once per VPL * 16 gathered bytes.
+template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, int EP>
 __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0,
                                             int chunk_end)
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
+    constexpr int UB = kLoads / VPL;                      // steps whose loads are issued together
+    constexpr int R = UB > LPR ? UB / LPR : 1;            // index registers per lane and batch
+    constexpr int SPB = R * LPR;                          // steps per batch
+    constexpr int EPB = R * S;                            // entries per batch
+    constexpr unsigned kFull = 0xffffffffu;
     const int tid = threadIdx.x;
     const int slot = block_in_range * ROWS + tid / S;
-    const int ls = tid % S;
-    const int g = ls / LPR;
-    const int j = col0 + (ls % LPR) * VECN;
-    const bool col_ok = j < chunk_end;
+    const int sl = tid % S;
+    const int g = sl / LPR;
+    const int c = sl % LPR;
     const bool active = slot < rg.item_count;
+
+    int jq[VPL];
+    bool okq[VPL];
+    const T* xq[VPL];
+#pragma unroll
+    for (int q = 0; q < VPL; ++q) {
+        jq[q] = col0 + (c + q * LPR) * VECN;
+        okq[q] = jq[q] < chunk_end;
+        xq[q] = static_cast<const T*>(a.x) + (okq[q] ? jq[q] : col0);   // out-of-chunk lanes re-read a valid column
+    }
 
     int32_t row = 0, b = 0, e = 0;
     if (active) {
@@ -100,80 +121,116 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         }
     }
 
-    float acc[VECN];
+    float acc[VPL][VECN];
 #pragma unroll
-    for (int i = 0; i < VECN; ++i) acc[i] = 0.f;
-    const T* xj = static_cast<const T*>(a.x) + j;
+    for (int q = 0; q < VPL; ++q)
+#pragma unroll
+        for (int i = 0; i < VECN; ++i) acc[q][i] = 0.f;
 
-    // Software pipeline: the indices (and weights) of step i+1 are requested right after the feature
-    // loads of step i are issued, so the index stream from HBM overlaps the gathers from L2.
-    int32_t u[kUnroll];
-    float w[kUnroll];
+    const uint32_t ld = (uint32_t)a.ldx;
+    const int n_batches = __reduce_max_sync(kFull, (e - b + EPB - 1) / EPB);     // the warp loops together
+
+    int32_t ucur[R];
+    float wcur[R];
 #pragma unroll
-    for (int t = 0; t < kUnroll; ++t) {
-        const int32_t kk = b + g + t * EP;
+    for (int r = 0; r < R; ++r) {
+        const int32_t kk = b + r * S + sl;
         const bool ok = kk < e;
-        u[t] = ok ? __ldcs(a.col_idx + kk) : -1;
-        if (WEIGHTED) w[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
+        ucur[r] = ok ? __ldcs(a.col_idx + kk) : -1;
+        wcur[r] = (WEIGHTED && ok) ? __ldcs(a.edge_w + kk) : 0.f;
     }
-    for (int32_t k = b + g; k < e; k += EP * kUnroll) {
-        Vec<T, VECN> v[kUnroll];
+
+    for (int ib = 0; ib < n_batches; ++ib) {
+        const int32_t kb = b + ib * EPB;
+        // the next batch's indices are requested before this batch's gathers are consumed
+        int32_t unext[R];
+        float wnext[R];
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            if (u[t] >= 0 && col_ok) v[t].load(xj + (int64_t)u[t] * a.ldx);
-            else v[t].zero();
-        }
-        int32_t un[kUnroll];
-        float wn[kUnroll];
-#pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            const int32_t kk = k + (kUnroll + t) * EP;
+        for (int r = 0; r < R; ++r) {
+            const int32_t kk = kb + EPB + r * S + sl;
             const bool ok = kk < e;
-            un[t] = ok ? __ldcs(a.col_idx + kk) : -1;
-            if (WEIGHTED) wn[t] = ok ? __ldcs(a.edge_w + kk) : 0.f;
+            unext[r] = ok ? __ldcs(a.col_idx + kk) : -1;
+            wnext[r] = (WEIGHTED && ok) ? __ldcs(a.edge_w + kk) : 0.f;
         }
+        const bool full = __all_sync(kFull, kb + EPB <= e);
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
+        for (int s0 = 0; s0 < SPB; s0 += UB) {
+            Vec<T, VECN> v[UB][VPL];
+            float wv[UB];
+            if (full) {
 #pragma unroll
-            for (int i = 0; i < VECN; ++i) {
-                if (WEIGHTED) acc[i] = fmaf(w[t], v[t].get(i), acc[i]);
-                else acc[i] += v[t].get(i);
+                for (int i = 0; i < UB; ++i) {
+                    const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
+                    const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
+                    if (WEIGHTED) wv[i] = __shfl_sync(kFull, wcur[r], t * EP + g, S);
+                    const size_t off = (size_t)(uint32_t)u * ld;
+#pragma unroll
+                    for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < UB; ++i) {
+                    const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
+                    const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
+                    if (WEIGHTED) wv[i] = __shfl_sync(kFull, wcur[r], t * EP + g, S);
+                    const size_t off = (size_t)(uint32_t)max(u, 0) * ld;
+#pragma unroll
+                    for (int q = 0; q < VPL; ++q) {
+                        if (u >= 0) v[i][q].load(xq[q] + off);
+                        else v[i][q].zero();
+                    }
+                }
             }
-            u[t] = un[t];
-            if (WEIGHTED) w[t] = wn[t];
+#pragma unroll
+            for (int i = 0; i < UB; ++i)
+#pragma unroll
+                for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                    for (int k = 0; k < VECN; ++k) {
+                        if (WEIGHTED) acc[q][k] = fmaf(wv[i], v[i][q].get(k), acc[q][k]);
+                        else acc[q][k] += v[i][q].get(k);
+                    }
         }
+#pragma unroll
+        for (int r = 0; r < R; ++r) { ucur[r] = unext[r]; wcur[r] = wnext[r]; }
     }
 
     // fixed-order combination of the EP partial sums of the row
 #pragma unroll
-    for (int o = S / 2; o >= LPR; o >>= 1) {
+    for (int o = S / 2; o >= LPR; o >>= 1)
 #pragma unroll
-        for (int i = 0; i < VECN; ++i) acc[i] += __shfl_down_sync(0xffffffffu, acc[i], o, S);
-    }
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int i = 0; i < VECN; ++i) acc[q][i] += __shfl_down_sync(kFull, acc[q][i], o, S);
 
-    if (!active || g != 0 || !col_ok) return;
-    if (rg.hub) {
-        float* p = a.partial + (int64_t)slot * a.fpad + j;
+    if (!active || g != 0) return;
+    const float scale = (WEIGHTED || rg.hub) ? 1.f : a.rdeg[row];
 #pragma unroll
-        for (int i = 0; i < VECN; ++i)
-            if (j + i < chunk_end) p[i] = acc[i];
-        return;
-    }
-    const float scale = WEIGHTED ? 1.f : a.rdeg[row];
-    const int64_t o = (int64_t)row * a.ldo + j;
-    if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
+    for (int q = 0; q < VPL; ++q) {
+        if (!okq[q]) continue;
+        const int j = jq[q];
+        if (rg.hub) {
+            float* p = a.partial + (int64_t)slot * a.fpad + j;
 #pragma unroll
-        for (int i = 0; i < VECN; i += 4)
-            __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
-                   make_float4(acc[i] * scale, acc[i + 1] * scale, acc[i + 2] * scale, acc[i + 3] * scale));
-    } else {
+            for (int i = 0; i < VECN; ++i)
+                if (j + i < chunk_end) p[i] = acc[q][i];
+            continue;
+        }
+        const int64_t o = (int64_t)row * a.ldo + j;
+        if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
 #pragma unroll
-        for (int i = 0; i < VECN; ++i)
-            if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[i] * scale);
+            for (int i = 0; i < VECN; i += 4)
+                __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
+                       make_float4(acc[q][i] * scale, acc[q][i + 1] * scale, acc[q][i + 2] * scale, acc[q][i + 3] * scale));
+        } else {
+#pragma unroll
+            for (int i = 0; i < VECN; ++i)
+                if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[q][i] * scale);
+        }
     }
 }
 
-template <typename T, int VECN, int LPR, bool WEIGHTED>
+template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED>
 __global__ void __launch_bounds__(kBlock) gather_aggregate(const __grid_constant__ GatherArgs a)
 {
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
@@ -183,7 +240,7 @@ __global__ void __launch_bounds__(kBlock) gather_aggregate(const __grid_constant
     const int ctile = rem % a.n_ctiles;
     const int chunk_begin = chunk * a.chunk_width;
     const int chunk_end = min(a.f, chunk_begin + a.chunk_width);
-    const int col0 = chunk_begin + ctile * (LPR * VECN);
+    const int col0 = chunk_begin + ctile * (LPR * VPL * VECN);
     if (col0 >= chunk_end) return;
     int r = 0;
 #pragma unroll
@@ -192,12 +249,12 @@ __global__ void __launch_bounds__(kBlock) gather_aggregate(const __grid_constant
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gather_rows<T, VECN, LPR, WEIGHTED, 1>(a, rg, bir, col0, chunk_end); break;
-        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 2>(a, rg, bir, col0, chunk_end); break;
-        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 4>(a, rg, bir, col0, chunk_end); break;
-        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 8>(a, rg, bir, col0, chunk_end); break;
-        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, WEIGHTED, 16>(a, rg, bir, col0, chunk_end); break;
-        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, WEIGHTED, 32>(a, rg, bir, col0, chunk_end); break;
+        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end); break;
+        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end); break;
+        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end); break;
+        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end); break;
+        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end); break;
+        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end); break;
     }
 }
 
@@ -223,23 +280,24 @@ hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict__ hu
 typedef void (*GatherKernel)(const GatherArgs);
 
 template <typename T, int VECN, bool WEIGHTED>
-static GatherKernel pick_lpr(int lpr)
+static GatherKernel pick_lpr(int lpr, int vpl)
 {
+    if (vpl == 1) return gather_aggregate<T, VECN, 1, 1, WEIGHTED>;
     switch (lpr) {
-        case 1: return gather_aggregate<T, VECN, 1, WEIGHTED>;
-        case 2: return gather_aggregate<T, VECN, 2, WEIGHTED>;
-        case 4: return gather_aggregate<T, VECN, 4, WEIGHTED>;
-        case 8: return gather_aggregate<T, VECN, 8, WEIGHTED>;
-        case 16: return gather_aggregate<T, VECN, 16, WEIGHTED>;
-        default: return gather_aggregate<T, VECN, 32, WEIGHTED>;
+        case 1: return gather_aggregate<T, VECN, 1, 2, WEIGHTED>;
+        case 2: return gather_aggregate<T, VECN, 2, 2, WEIGHTED>;
+        case 4: return gather_aggregate<T, VECN, 4, 2, WEIGHTED>;
+        case 8: return gather_aggregate<T, VECN, 8, 2, WEIGHTED>;
+        case 16: return gather_aggregate<T, VECN, 16, 2, WEIGHTED>;
+        default: return gather_aggregate<T, VECN, 32, 2, WEIGHTED>;
     }
 }
 
 template <bool WEIGHTED>
-static GatherKernel pick_kernel(gnnfd_dtype_t xdt, bool vec, int lpr)
+static GatherKernel pick_kernel(gnnfd_dtype_t xdt, bool vec, int lpr, int vpl)
 {
-    if (xdt == GNNFD_F32) return vec ? pick_lpr<float, 4, WEIGHTED>(lpr) : pick_lpr<float, 1, WEIGHTED>(lpr);
-    return vec ? pick_lpr<__nv_bfloat16, 8, WEIGHTED>(lpr) : pick_lpr<__nv_bfloat16, 1, WEIGHTED>(lpr);
+    if (xdt == GNNFD_F32) return vec ? pick_lpr<float, 4, WEIGHTED>(lpr, vpl) : pick_lpr<float, 1, WEIGHTED>(lpr, vpl);
+    return vec ? pick_lpr<__nv_bfloat16, 8, WEIGHTED>(lpr, vpl) : pick_lpr<__nv_bfloat16, 1, WEIGHTED>(lpr, vpl);
 }
 
 static size_t partial_bytes(const gnnfd_csr_t* csr, int32_t f)
@@ -252,7 +310,8 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
                      int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width, void* d_scratch,
                      size_t scratch_bytes, cudaStream_t s)
 {
-    if (!csr || !d_x || !d_out || f <= 0 || chunk_width <= 0 || ldx < f || ldo < f) return GNNFD_INVALID_ARG;
+    if (!csr || !d_x || !d_out || f <= 0 || chunk_width <= 0 || ldx < f || ldo < f || ldx > 0x7fffffffll)
+        return GNNFD_INVALID_ARG;
     if ((xdt != GNNFD_F32 && xdt != GNNFD_BF16) || (odt != GNNFD_F32 && odt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
     const size_t need = partial_bytes(csr, f);
     if (need > 0 && (!d_scratch || scratch_bytes < need)) return GNNFD_WORKSPACE_TOO_SMALL;
@@ -265,16 +324,18 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
     // 128-bit loads need 16-byte aligned row starts and chunk starts
     const bool vec = ((uintptr_t)d_x % 16 == 0) && ((ldx * xsize) % 16 == 0) && (n_chunks == 1 || cw % vecn == 0);
     const int elems = vec ? vecn : 1;
-    int lanes = (cw + elems - 1) / elems;
+    // a lane covers two vectors of the chunk unless the chunk is a single vector wide
+    const int vectors = (cw + elems - 1) / elems;
+    const int vpl = vectors > 1 ? 2 : 1;
     int lpr = 1;
-    while (lpr < lanes && lpr < 32) lpr <<= 1;
+    while (lpr * vpl < vectors && lpr < 32) lpr <<= 1;
 
     GatherArgs a;
     a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.edge_w = csr->edge_w; a.rdeg = csr->rdeg;
     a.row_order = csr->row_order; a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin;
     a.x = d_x; a.out = d_out; a.partial = static_cast<float*>(d_scratch);
     a.ldx = ldx; a.ldo = ldo; a.f = f; a.chunk_width = cw;
-    a.n_ctiles = (cw + lpr * elems - 1) / (lpr * elems);
+    a.n_ctiles = (cw + lpr * vpl * elems - 1) / (lpr * vpl * elems);
     a.fpad = (int32_t)align_up((size_t)f, 4);
     a.out_bf16 = odt == GNNFD_BF16;
     a.out_vec_ok = odt == GNNFD_F32 && ((uintptr_t)d_out % 16 == 0) && (ldo % 4 == 0) && (n_chunks == 1 || cw % 4 == 0);
@@ -285,7 +346,7 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
     if (grid > 0x7fffffffll || blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
 
     if (grid > 0) {
-        GatherKernel kernel = weighted ? pick_kernel<true>(xdt, vec, lpr) : pick_kernel<false>(xdt, vec, lpr);
+        GatherKernel kernel = weighted ? pick_kernel<true>(xdt, vec, lpr, vpl) : pick_kernel<false>(xdt, vec, lpr, vpl);
         GNNFD_LAUNCH(weighted ? "gather_aggregate_gcn" : "gather_aggregate_sage", s, kernel, (unsigned)grid, kBlock, 0, a);
     }
     const int64_t n_hub = csr->bin_count[4];

@@ -251,25 +251,43 @@ row_pointers(const u64* __restrict__ keys, BuildCounts* __restrict__ counts, int
     row_ptr[v] = lo;
 }
 
+// Degree class of a row: exact degree up to 8, then quarter octaves of (deg - 1) up to the hub
+// threshold, then one class for hub rows.  Classes are monotone in the degree, so each of the five
+// launch bins (<= 8, <= 32, <= 128, <= hub threshold, hub) is a contiguous range of classes.
+constexpr int kHubClass = 41;
+__device__ __forceinline__ int degree_class(int32_t deg)
+{
+    if (deg <= kBinDeg0) return deg;
+    if (deg > kBinDeg3) return kHubClass;
+    const int t = deg - 1;
+    const int o = 31 - __clz(t);                       // 3 .. 10
+    return 9 + (o - 3) * 4 + ((t >> (o - 2)) & 3);
+}
 __device__ __forceinline__ int degree_bin(int32_t deg)
 {
     return deg <= kBinDeg0 ? 0 : deg <= kBinDeg1 ? 1 : deg <= kBinDeg2 ? 2 : deg <= kBinDeg3 ? 3 : 4;
 }
 
-// degree normalisers (rounded once from fp64) and the bin membership flags, bin-major [5][n]
+// degree normalisers (rounded once from fp64), the bin sizes, and the (class, row) sort keys
 __global__ void __launch_bounds__(kThreads)
-degrees_and_bins(const int32_t* __restrict__ row_ptr, int64_t n, float* __restrict__ dinv, float* __restrict__ rdeg,
-                 int32_t* __restrict__ bin_flag, BuildCounts* __restrict__ counts)
+degrees_and_classes(const int32_t* __restrict__ row_ptr, int64_t n, float* __restrict__ dinv, float* __restrict__ rdeg,
+                    u64* __restrict__ class_keys, int32_t* __restrict__ class_vals, BuildCounts* __restrict__ counts)
 {
     const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     int32_t deg = 0;
+    int bin = -1;
     if (v < n) {
         deg = row_ptr[v + 1] - row_ptr[v];
         dinv[v] = deg > 0 ? (float)(1.0 / sqrt((double)deg)) : 0.f;
         rdeg[v] = deg > 0 ? (float)(1.0 / (double)deg) : 0.f;
-        const int bin = degree_bin(deg);
+        bin = degree_bin(deg);
+        class_keys[v] = ((u64)degree_class(deg) << 32) | (u64)v;
+        class_vals[v] = (int32_t)v;
+    }
 #pragma unroll
-        for (int b = 0; b < kNumBins; ++b) bin_flag[(int64_t)b * n + v] = b == bin ? 1 : 0;
+    for (int b = 0; b < kNumBins; ++b) {
+        const int c = __syncthreads_count(bin == b);
+        if (threadIdx.x == 0 && c) atomicAdd(&counts->bin_count[b], c);
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) deg = max(deg, __shfl_xor_sync(0xffffffffu, deg, o));
@@ -290,24 +308,6 @@ finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals,
     __stcs(col_idx + k, s);
     __stcs(edge_w + k, __ldg(dinv + s) * __ldg(dinv + d));
     if (vals) __stcs(perm + k, __ldcs(vals + k));
-}
-
-__global__ void __launch_bounds__(kThreads)
-place_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ bin_pos, int64_t n,
-           int32_t* __restrict__ row_order, BuildCounts* __restrict__ counts)
-{
-    const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (v < n) {
-        const int bin = degree_bin(row_ptr[v + 1] - row_ptr[v]);
-        row_order[bin_pos[(int64_t)bin * n + v]] = (int32_t)v;
-    }
-    if (v == 0) {
-        for (int b = 0; b < kNumBins; ++b) {
-            const int32_t start = bin_pos[(int64_t)b * n];
-            const int32_t end = b + 1 < kNumBins ? bin_pos[(int64_t)(b + 1) * n] : (int32_t)n;
-            counts->bin_count[b] = end - start;
-        }
-    }
 }
 
 // segments per hub row; entry n_hub (one past the end) is 0 so that the scan yields the total
@@ -348,7 +348,8 @@ fill_segments(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ r
 
 struct BuildLayout {
     int64_t m;             // candidate edges
-    int64_t n_tiles;       // sort tiles
+    int64_t n_tiles;       // sort tiles of the edge sort
+    int64_t row_tiles;     // sort tiles of the row (degree class) sort
     int64_t hub_cap;       // upper bound on hub rows
     int64_t seg_cap;       // upper bound on hub segments
     int src_bits, key_bits, passes, digit_bits;
@@ -367,6 +368,7 @@ static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
     L->m = m;
     L->n_tiles = (m + kSortTile - 1) / kSortTile;
     if (L->n_tiles == 0) L->n_tiles = 1;
+    L->row_tiles = (n + kSortTile - 1) / kSortTile;
     L->hub_cap = m / (GNNFD_HUB_DEGREE + 1) + 1;
     L->seg_cap = m / kHubSegment + L->hub_cap + 1;
     int bits = 1;
@@ -409,19 +411,20 @@ struct ScratchPtrs {
 
 static size_t flag_ints(int64_t n, const BuildLayout& L)
 {
-    size_t a = (size_t)L.m, b = (size_t)kNumBins * (size_t)n, c = (size_t)L.hub_cap + 1;
+    // dedup flags (m), a 64-bit dump for the row sort's keys (2 ints per row), hub segment counts
+    size_t a = (size_t)L.m, b = 2 * (size_t)n + 2, c = (size_t)L.hub_cap + 1;
     size_t r = a > b ? a : b;
     return (r > c ? r : c) + 1;
 }
 
 static void carve_scratch(Carver& c, int64_t n, const BuildLayout& L, ScratchPtrs* p)
 {
-    const size_t cap = (size_t)(L.m > 0 ? L.m : 1);
+    const size_t cap = (size_t)(L.m > n ? L.m : n);      // the row sort reuses the edge sort's buffers
     p->keys_a = c.take<u64>(cap);
     p->keys_b = c.take<u64>(cap);
     p->vals_a = c.take<int32_t>(cap);
     p->vals_b = c.take<int32_t>(cap);
-    const size_t hist_ints = (size_t)kRadix * (size_t)L.n_tiles;
+    const size_t hist_ints = (size_t)kRadix * (size_t)(L.n_tiles > L.row_tiles ? L.n_tiles : L.row_tiles);
     p->hist = c.take<int32_t>(hist_ints);
     const size_t fl = flag_ints(n, L);
     p->flags = c.take<int32_t>(fl);
@@ -518,22 +521,30 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
             if (rc) return rc;
             GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys, vals, S.flags,
                          pos, m, keys_alt, P.perm, P.counts);
-            keys = keys_alt;
+            u64* tk = keys; keys = keys_alt; keys_alt = tk;
         }
     }
     GNNFD_LAUNCH("row_pointers", s, row_pointers, blocks_for((size_t)n + 1, kThreads), kThreads, 0, keys, P.counts, n,
                  L.src_bits, dedup ? 1 : 0, P.row_ptr);
-    GNNFD_LAUNCH("degrees_and_bins", s, degrees_and_bins, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
-                 P.dinv, P.rdeg, S.flags, P.counts);
+    // keys_alt / vals_alt are free from here on: they take the (degree class, row) pairs
+    GNNFD_LAUNCH("degrees_and_classes", s, degrees_and_classes, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
+                 P.dinv, P.rdeg, keys_alt, vals_alt, P.counts);
     if (m > 0)
         GNNFD_LAUNCH("finalize_entries", s, finalize_entries, blocks_for(m, kThreads), kThreads, 0, keys,
                      dedup ? (const int32_t*)nullptr : (const int32_t*)vals, P.counts, L.src_bits, P.dinv, P.col_idx,
                      P.edge_w, P.perm, m);
-    rc = exclusive_scan_i32(S.flags, S.flags, (size_t)kNumBins * (size_t)n, S.scan_temp, s);
-    if (rc) return rc;
-    GNNFD_LAUNCH("place_rows", s, place_rows, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, S.flags, n,
-                 P.row_order, P.counts);
-    // the bin positions are consumed; reuse the flag buffer for the per-hub-row segment counts
+    // row_order = rows sorted by degree class, ascending row id inside a class: one stable radix pass
+    {
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)sizeof(ScatterSmem)));
+        GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.row_tiles, kThreads, 0, keys_alt, n, 32, kRadix - 1,
+                     L.row_tiles, S.hist);
+        rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.row_tiles, S.scan_temp, s);
+        if (rc) return rc;
+        GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.row_tiles, kThreads, sizeof(ScatterSmem), keys_alt,
+                     vals_alt, reinterpret_cast<u64*>(S.flags), P.row_order, n, 32, kRadix - 1, L.row_tiles, S.hist);
+    }
+    // the flag buffer is free again: per-hub-row segment counts
     int32_t* seg_count = S.flags;
     GNNFD_LAUNCH("hub_segment_counts", s, hub_segment_counts, blocks_for((size_t)L.hub_cap + 1, kThreads), kThreads, 0,
                  P.row_ptr, P.row_order, n, P.counts, L.hub_cap, seg_count);

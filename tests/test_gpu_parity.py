@@ -65,18 +65,32 @@ def check_csr(g, n, src, dst, flags):
     return csr, (row_ptr, col, perm)
 
 
+def degree_class(deg, hub_degree):
+    """Fine degree classes of the launch schedule: exact degree up to 8, quarter octaves of deg - 1 up to
+    the hub threshold, one class for hub rows (restated from the header's description)."""
+    deg = np.asarray(deg, np.int64)
+    t = np.maximum(deg - 1, 8)
+    o = np.floor(np.log2(t)).astype(np.int64)
+    mid = 9 + (o - 3) * 4 + ((t >> (o - 2)) & 3)
+    return np.where(deg <= 8, deg, np.where(deg > hub_degree, 41, mid))
+
+
 def check_schedule(g, csr, deg):
     order = csr.row_order.cpu().numpy()
     n = len(deg)
     assert sorted(order.tolist()) == list(range(n))
     bounds = [8, 32, 128, g.HUB_DEGREE]
     bins = np.searchsorted(bounds, deg, side="left")          # first bound >= deg; 4 = hub
+    cls = degree_class(deg, g.HUB_DEGREE)
     start = 0
     for b in range(5):
         part = order[start:start + csr.bin_count[b]]
-        assert (bins[part] == b).all() and (np.diff(part) > 0).all()
+        assert (bins[part] == b).all()
         start += csr.bin_count[b]
     assert start == n
+    # rows are ordered by (class, row id)
+    key = cls[order] * (n + 1) + order
+    assert (np.diff(key) > 0).all()
     hubs = order[n - csr.bin_count[4]:]
     seg_ptr = csr.hub_seg_ptr.cpu().numpy()
     seg_row = csr.seg_row.cpu().numpy()
