@@ -1,5 +1,4 @@
-// GAT: attention scores, the fused logit + online-softmax + weighted-sum aggregation, and the
-// materialised edge softmax.
+// GAT: attention scores and the fused logit + online-softmax + weighted-sum aggregation.
 //
 // The attention logits always use the full head width (scores are computed once from all of z);
 // feature decomposition only cuts the weighted sum into column chunks, so the chunked result equals
@@ -103,19 +102,38 @@ gat_scores(const T* __restrict__ z, int64_t ldz, const float* __restrict__ a_src
 
 // ------------------------------------------------------------------ fused aggregation
 
-template <typename T, int VECN, int LPR, int EP>
+constexpr int kLoads = 8;      // 16-byte feature loads kept in flight per lane
+
+// One row (or hub segment) per S = LPR * EP lanes, same batching as the GCN / SAGE gather: the S lanes
+// fetch S column indices per round with one coalesced load and pass them on by shuffle.  A lane
+// covers VPL adjacent vectors, all inside one head, so it needs one logit per entry.
+template <typename T, int VECN, int LPR, int VPL, int EP>
 __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int block_in_range, int col0, int chunk_end)
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
+    constexpr int UB = kLoads / VPL;
+    constexpr int R = UB > LPR ? UB / LPR : 1;
+    constexpr int SPB = R * LPR;
+    constexpr int EPB = R * S;
+    constexpr unsigned kFull = 0xffffffffu;
     const int tid = threadIdx.x;
     const int slot = block_in_range * ROWS + tid / S;
-    const int ls = tid % S;
-    const int g = ls / LPR;
-    const int j = col0 + (ls % LPR) * VECN;
-    const bool col_ok = j < chunk_end;
+    const int sl = tid % S;
+    const int g = sl / LPR;
+    const int c = sl % LPR;
+    const int j0 = col0 + c * (VPL * VECN);
     const bool active = slot < rg.item_count;
-    const int h = col_ok ? j / a.dim : 0;      // all VECN columns of a lane lie in one head
+    const bool lane_ok = j0 < chunk_end;
+    const int h = (lane_ok ? j0 : col0) / a.dim;
+
+    bool okq[VPL];
+    const T* zq[VPL];
+#pragma unroll
+    for (int q = 0; q < VPL; ++q) {
+        okq[q] = j0 + q * VECN < chunk_end;
+        zq[q] = static_cast<const T*>(a.z) + (okq[q] ? j0 + q * VECN : col0);
+    }
 
     int32_t row = 0, b = 0, e = 0;
     if (active) {
@@ -131,91 +149,126 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
     }
     const float sd = active ? a.s_dst[(int64_t)row * a.heads + h] : 0.f;
     const float* ssrc = a.s_src + h;
-    const T* zj = static_cast<const T*>(a.z) + j;
+    const uint32_t ld = (uint32_t)a.ldz;
+    const uint32_t heads = (uint32_t)a.heads;
 
     float m = -CUDART_INF_F, l = 0.f;
-    float acc[VECN];
+    float acc[VPL][VECN];
 #pragma unroll
-    for (int i = 0; i < VECN; ++i) acc[i] = 0.f;
+    for (int q = 0; q < VPL; ++q)
+#pragma unroll
+        for (int i = 0; i < VECN; ++i) acc[q][i] = 0.f;
 
-    for (int32_t k = b + g; k < e; k += EP * kUnroll) {
-        int32_t u[kUnroll];
+    const int n_batches = __reduce_max_sync(kFull, (e - b + EPB - 1) / EPB);
+    int32_t ucur[R];
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            const int32_t kk = k + t * EP;
-            u[t] = kk < e ? __ldcs(a.col_idx + kk) : -1;
+    for (int r = 0; r < R; ++r) {
+        const int32_t kk = b + r * S + sl;
+        ucur[r] = kk < e ? __ldcs(a.col_idx + kk) : -1;
+    }
+
+    for (int ib = 0; ib < n_batches; ++ib) {
+        const int32_t kb = b + ib * EPB;
+        int32_t unext[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int32_t kk = kb + EPB + r * S + sl;
+            unext[r] = kk < e ? __ldcs(a.col_idx + kk) : -1;
         }
-        float logit[kUnroll];
-        ZVec<T, VECN> v[kUnroll];
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            if (u[t] >= 0) {
-                logit[t] = __ldg(ssrc + (int64_t)u[t] * a.heads);
-                if (col_ok) v[t].load(zj + (int64_t)u[t] * a.ldz); else v[t].zero();
-            } else {
-                logit[t] = 0.f;
-                v[t].zero();
+        for (int s0 = 0; s0 < SPB; s0 += UB) {
+            ZVec<T, VECN> v[UB][VPL];
+            float lg[UB];
+            bool valid[UB];
+#pragma unroll
+            for (int i = 0; i < UB; ++i) {
+                const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
+                const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
+                valid[i] = u >= 0;
+                const uint32_t uu = (uint32_t)max(u, 0);
+                lg[i] = valid[i] ? __ldg(ssrc + (size_t)uu * heads) : 0.f;
+                const size_t off = (size_t)uu * ld;
+#pragma unroll
+                for (int q = 0; q < VPL; ++q) {
+                    if (valid[i]) v[i][q].load(zq[q] + off);
+                    else v[i][q].zero();
+                }
+            }
+            float mx = m;
+#pragma unroll
+            for (int i = 0; i < UB; ++i) {
+                lg[i] = leaky(lg[i] + sd, a.slope);
+                if (valid[i]) mx = fmaxf(mx, lg[i]);
+            }
+            const float rescale = merge_scale(m, mx);
+            m = mx;
+            l *= rescale;
+#pragma unroll
+            for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                for (int i = 0; i < VECN; ++i) acc[q][i] *= rescale;
+#pragma unroll
+            for (int i = 0; i < UB; ++i) {
+                const float p = valid[i] ? expf(lg[i] - m) : 0.f;
+                l += p;
+#pragma unroll
+                for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                    for (int k = 0; k < VECN; ++k) acc[q][k] = fmaf(p, v[i][q].get(k), acc[q][k]);
             }
         }
-        float mx = m;
 #pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            logit[t] = leaky(logit[t] + sd, a.slope);
-            if (u[t] >= 0) mx = fmaxf(mx, logit[t]);
-        }
-        const float rescale = merge_scale(m, mx);     // the first edge of the step is valid, so mx is finite
-        m = mx;
-        l *= rescale;
-#pragma unroll
-        for (int i = 0; i < VECN; ++i) acc[i] *= rescale;
-#pragma unroll
-        for (int t = 0; t < kUnroll; ++t) {
-            const float p = u[t] >= 0 ? expf(logit[t] - m) : 0.f;
-            l += p;
-#pragma unroll
-            for (int i = 0; i < VECN; ++i) acc[i] = fmaf(p, v[t].get(i), acc[i]);
-        }
+        for (int r = 0; r < R; ++r) ucur[r] = unext[r];
     }
 
     // merge the EP groups of the row, fixed tree
 #pragma unroll
     for (int o = S / 2; o >= LPR; o >>= 1) {
-        const float m2 = __shfl_down_sync(0xffffffffu, m, o, S);
-        const float l2 = __shfl_down_sync(0xffffffffu, l, o, S);
+        const float m2 = __shfl_down_sync(kFull, m, o, S);
+        const float l2 = __shfl_down_sync(kFull, l, o, S);
         const float mn = fmaxf(m, m2);
         const float sa = merge_scale(m, mn), sb = merge_scale(m2, mn);
         l = l * sa + l2 * sb;
 #pragma unroll
-        for (int i = 0; i < VECN; ++i) {
-            const float a2 = __shfl_down_sync(0xffffffffu, acc[i], o, S);
-            acc[i] = acc[i] * sa + a2 * sb;
-        }
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int i = 0; i < VECN; ++i) {
+                const float a2 = __shfl_down_sync(kFull, acc[q][i], o, S);
+                acc[q][i] = acc[q][i] * sa + a2 * sb;
+            }
         m = mn;
     }
 
-    if (!active || g != 0 || !col_ok) return;
+    if (!active || g != 0 || !lane_ok) return;
     if (rg.hub) {
-        float* p = a.partial + (int64_t)slot * a.fpad + j;
-#pragma unroll
-        for (int i = 0; i < VECN; ++i)
-            if (j + i < chunk_end) p[i] = acc[i];
         // every lane of a head holds the same (m, l); the first lane of each head inside this column tile stores
         // it (sweeps that share a head store identical values)
-        if (j % a.dim == 0 || ls % LPR == 0) {
+        if (j0 % a.dim == 0 || c == 0) {
             float* ml = a.partial_ml + ((int64_t)slot * a.heads + h) * 2;
             ml[0] = m;
             ml[1] = l;
         }
-        return;
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
-    const int64_t o = (int64_t)row * a.ldo + j;
 #pragma unroll
-    for (int i = 0; i < VECN; ++i)
-        if (j + i < chunk_end) store_out(a.out, a.out_bf16, o + i, acc[i] * inv);
+    for (int q = 0; q < VPL; ++q) {
+        if (!okq[q]) continue;
+        const int j = j0 + q * VECN;
+        if (rg.hub) {
+            float* p = a.partial + (int64_t)slot * a.fpad + j;
+#pragma unroll
+            for (int i = 0; i < VECN; ++i)
+                if (j + i < chunk_end) p[i] = acc[q][i];
+        } else {
+            const int64_t o = (int64_t)row * a.ldo + j;
+#pragma unroll
+            for (int i = 0; i < VECN; ++i)
+                if (j + i < chunk_end) store_out(a.out, a.out_bf16, o + i, acc[q][i] * inv);
+        }
+    }
 }
 
-template <typename T, int VECN, int LPR>
+template <typename T, int VECN, int LPR, int VPL>
 __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ GatArgs a)
 {
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
@@ -225,7 +278,7 @@ __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ 
     const int ctile = rem % a.n_ctiles;
     const int chunk_begin = chunk * a.chunk_width;
     const int chunk_end = min(a.f, chunk_begin + a.chunk_width);
-    const int col0 = chunk_begin + ctile * (LPR * VECN);
+    const int col0 = chunk_begin + ctile * (LPR * VPL * VECN);
     if (col0 >= chunk_end) return;
     int r = 0;
 #pragma unroll
@@ -234,12 +287,12 @@ __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ 
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gat_rows<T, VECN, LPR, 1>(a, rg, bir, col0, chunk_end); break;
-        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, 2>(a, rg, bir, col0, chunk_end); break;
-        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, 4>(a, rg, bir, col0, chunk_end); break;
-        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, 8>(a, rg, bir, col0, chunk_end); break;
-        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, 16>(a, rg, bir, col0, chunk_end); break;
-        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, 32>(a, rg, bir, col0, chunk_end); break;
+        case 0: gat_rows<T, VECN, LPR, VPL, 1>(a, rg, bir, col0, chunk_end); break;
+        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, VPL, 2>(a, rg, bir, col0, chunk_end); break;
+        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, VPL, 4>(a, rg, bir, col0, chunk_end); break;
+        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, VPL, 8>(a, rg, bir, col0, chunk_end); break;
+        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, VPL, 16>(a, rg, bir, col0, chunk_end); break;
+        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, VPL, 32>(a, rg, bir, col0, chunk_end); break;
     }
 }
 
@@ -267,111 +320,27 @@ gat_hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict_
     store_out(out, out_bf16, (int64_t)row * ldo + j, den > 0.f ? num / den : 0.f);
 }
 
-// ------------------------------------------------------------------ edge softmax
-//
-// GROUP threads (a warp, or a whole block for hub rows) share a row.  When heads is a power of two
-// <= 32 a thread owns head t % heads and every (32 / heads)-th ... edge, so that alpha is written
-// with consecutive threads on consecutive addresses; otherwise the heads are taken one at a time.
-
-template <int GROUP>
-__device__ __forceinline__ float group_max(float v, int lanes_per_value, float* smem)
-{
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1)
-        if (o >= lanes_per_value) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    if (GROUP > 32) {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        __syncthreads();
-        smem[warp * 32 + lane] = v;
-        __syncthreads();
-        v = smem[lane];
-#pragma unroll
-        for (int w = 1; w < GROUP / 32; ++w) v = fmaxf(v, smem[w * 32 + lane]);
-    }
-    return v;
-}
-
-template <int GROUP>
-__device__ __forceinline__ float group_sum(float v, int lanes_per_value, float* smem)
-{
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1)
-        if (o >= lanes_per_value) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (GROUP > 32) {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        __syncthreads();
-        smem[warp * 32 + lane] = v;
-        __syncthreads();
-        v = smem[lane];
-#pragma unroll
-        for (int w = 1; w < GROUP / 32; ++w) v += smem[w * 32 + lane];
-    }
-    return v;
-}
-
-template <int GROUP>
-__device__ __forceinline__ void softmax_row(const int32_t* __restrict__ col_idx, const float* __restrict__ s_src,
-                                            const float* __restrict__ s_dst, int32_t row, int32_t b, int32_t e, int heads,
-                                            float slope, float* __restrict__ alpha, float* smem)
-{
-    const int t = threadIdx.x % GROUP;
-    const bool packed = heads <= 32 && (heads & (heads - 1)) == 0;
-    const int hh = packed ? heads : 1;           // heads handled together
-    const int step = GROUP / hh;                 // edges handled together
-    for (int h0 = 0; h0 < heads; h0 += hh) {
-        const int h = h0 + (t % hh);
-        const float sd = s_dst[(int64_t)row * heads + h];
-        float m = -CUDART_INF_F;
-        for (int32_t k = b + t / hh; k < e; k += step)
-            m = fmaxf(m, leaky(__ldg(s_src + (int64_t)col_idx[k] * heads + h) + sd, slope));
-        m = group_max<GROUP>(m, hh, smem);
-        float l = 0.f;
-        for (int32_t k = b + t / hh; k < e; k += step)
-            l += expf(leaky(__ldg(s_src + (int64_t)col_idx[k] * heads + h) + sd, slope) - m);
-        l = group_sum<GROUP>(l, hh, smem);
-        const float inv = 1.f / l;
-        for (int32_t k = b + t / hh; k < e; k += step)
-            __stcs(alpha + (int64_t)k * heads + h,
-                   expf(leaky(__ldg(s_src + (int64_t)col_idx[k] * heads + h) + sd, slope) - m) * inv);
-    }
-}
-
-__global__ void __launch_bounds__(kBlock)
-edge_softmax_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                  const int32_t* __restrict__ row_order, int64_t n_rows, const float* __restrict__ s_src,
-                  const float* __restrict__ s_dst, int heads, float slope, float* __restrict__ alpha)
-{
-    const int64_t slot = (int64_t)blockIdx.x * (kBlock / 32) + (threadIdx.x >> 5);
-    if (slot >= n_rows) return;               // whole warps leave together
-    const int32_t row = row_order[slot];
-    softmax_row<32>(col_idx, s_src, s_dst, row, row_ptr[row], row_ptr[row + 1], heads, slope, alpha, nullptr);
-}
-
-__global__ void __launch_bounds__(kBlock)
-edge_softmax_hubs(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                  const int32_t* __restrict__ hub_rows, const float* __restrict__ s_src, const float* __restrict__ s_dst,
-                  int heads, float slope, float* __restrict__ alpha)
-{
-    __shared__ float smem[kBlock];
-    const int32_t row = hub_rows[blockIdx.x];
-    softmax_row<kBlock>(col_idx, s_src, s_dst, row, row_ptr[row], row_ptr[row + 1], heads, slope, alpha, smem);
-}
-
 // ------------------------------------------------------------------ host side
 
 typedef void (*GatKernel)(const GatArgs);
 
-template <typename T, int VECN>
+template <typename T, int VECN, int VPL>
 static GatKernel pick_lpr(int lpr)
 {
     switch (lpr) {
-        case 1: return gat_aggregate<T, VECN, 1>;
-        case 2: return gat_aggregate<T, VECN, 2>;
-        case 4: return gat_aggregate<T, VECN, 4>;
-        case 8: return gat_aggregate<T, VECN, 8>;
-        case 16: return gat_aggregate<T, VECN, 16>;
-        default: return gat_aggregate<T, VECN, 32>;
+        case 1: return gat_aggregate<T, VECN, 1, VPL>;
+        case 2: return gat_aggregate<T, VECN, 2, VPL>;
+        case 4: return gat_aggregate<T, VECN, 4, VPL>;
+        case 8: return gat_aggregate<T, VECN, 8, VPL>;
+        case 16: return gat_aggregate<T, VECN, 16, VPL>;
+        default: return gat_aggregate<T, VECN, 32, VPL>;
     }
+}
+
+template <typename T, int VECN>
+static GatKernel pick_vpl(int lpr, int vpl)
+{
+    return vpl == 2 ? pick_lpr<T, VECN, 2>(lpr) : pick_lpr<T, VECN, 1>(lpr);
 }
 
 struct GatScratch {
@@ -435,7 +404,7 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     using namespace gnnfd;
     if (!csr || !d_z || !d_a_src || !d_a_dst || !d_out || heads <= 0 || dim <= 0 || chunk_width <= 0) return GNNFD_INVALID_ARG;
     const int64_t f64 = (int64_t)heads * dim;
-    if (f64 > 0x7fffffffll || ldz < f64 || ldo < f64) return GNNFD_INVALID_ARG;
+    if (f64 > 0x7fffffffll || ldz < f64 || ldo < f64 || ldz > 0x7fffffffll) return GNNFD_INVALID_ARG;
     if ((zdt != GNNFD_F32 && zdt != GNNFD_BF16) || (odt != GNNFD_F32 && odt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
     if (!d_scratch || ((uintptr_t)d_scratch & 255u)) return GNNFD_INVALID_ARG;
     const int32_t f = (int32_t)f64;
@@ -456,9 +425,11 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     const bool vec = ((uintptr_t)d_z % 16 == 0) && ((ldz * zsize) % 16 == 0) && (n_chunks == 1 || cw % vecn == 0) &&
                      (dim % vecn == 0);
     const int elems = vec ? vecn : 1;
-    const int lanes = (cw + elems - 1) / elems;
+    // a lane covers two adjacent vectors when both stay inside one head and chunks start on such pairs
+    const int vectors = (cw + elems - 1) / elems;
+    const int vpl = (vectors > 1 && dim % (2 * elems) == 0 && (n_chunks == 1 || cw % (2 * elems) == 0)) ? 2 : 1;
     int lpr = 1;
-    while (lpr < lanes && lpr < 32) lpr <<= 1;
+    while (lpr * vpl < vectors && lpr < 32) lpr <<= 1;
 
     GatArgs a;
     a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.row_order = csr->row_order;
@@ -467,7 +438,7 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     a.partial = g.partial; a.partial_ml = g.partial_ml;
     a.ldz = ldz; a.ldo = ldo; a.slope = negative_slope;
     a.f = f; a.heads = heads; a.dim = dim; a.chunk_width = cw;
-    a.n_ctiles = (cw + lpr * elems - 1) / (lpr * elems);
+    a.n_ctiles = (cw + lpr * vpl * elems - 1) / (lpr * vpl * elems);
     a.fpad = (int32_t)align_up((size_t)f, 4);
     a.out_bf16 = odt == GNNFD_BF16;
 
@@ -477,8 +448,8 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     if (grid > 0x7fffffffll || blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
     if (grid > 0) {
         GatKernel kernel;
-        if (zdt == GNNFD_F32) kernel = vec ? pick_lpr<float, 4>(lpr) : pick_lpr<float, 1>(lpr);
-        else kernel = vec ? pick_lpr<__nv_bfloat16, 8>(lpr) : pick_lpr<__nv_bfloat16, 1>(lpr);
+        if (zdt == GNNFD_F32) kernel = vec ? pick_vpl<float, 4>(lpr, vpl) : pick_vpl<float, 1>(lpr, vpl);
+        else kernel = vec ? pick_vpl<__nv_bfloat16, 8>(lpr, vpl) : pick_vpl<__nv_bfloat16, 1>(lpr, vpl);
         GNNFD_LAUNCH("gat_aggregate", s, kernel, (unsigned)grid, kBlock, 0, a);
     }
     const int64_t n_hub = csr->bin_count[4];
@@ -487,26 +458,6 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
         GNNFD_LAUNCH("gat_hub_reduce", s, gat_hub_reduce, gr, kBlock, 0, csr->row_order, csr->hub_seg_ptr, g.partial,
                      g.partial_ml, csr->bin_start[4], (int32_t)n_hub, f, a.fpad, heads, dim, d_out, ldo, a.out_bf16);
     }
-    GNNFD_CUDA_CHECK(cudaGetLastError());
-    return GNNFD_OK;
-}
-
-int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
-                       float negative_slope, float* d_alpha, void* stream)
-{
-    using namespace gnnfd;
-    if (!csr || !d_s_src || !d_s_dst || !d_alpha || heads <= 0) return GNNFD_INVALID_ARG;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int64_t n_hub = csr->bin_count[4];
-    const int64_t n_rows = csr->n - n_hub;      // the hub rows are the tail of row_order
-    if (n_rows > 0) {
-        const unsigned grid = (unsigned)((n_rows + kBlock / 32 - 1) / (kBlock / 32));
-        GNNFD_LAUNCH("edge_softmax_rows", s, edge_softmax_rows, grid, kBlock, 0, csr->row_ptr, csr->col_idx, csr->row_order,
-                     n_rows, d_s_src, d_s_dst, heads, negative_slope, d_alpha);
-    }
-    if (n_hub > 0)
-        GNNFD_LAUNCH("edge_softmax_hubs", s, edge_softmax_hubs, (unsigned)n_hub, kBlock, 0, csr->row_ptr, csr->col_idx,
-                     csr->row_order + csr->bin_start[4], d_s_src, d_s_dst, heads, negative_slope, d_alpha);
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
 }

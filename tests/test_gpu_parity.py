@@ -324,3 +324,27 @@ def test_gat_bf16_features(g):
     for width in (8, 32, 2):
         got = g.aggregate_gat(csr, zd, dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
         assert_close_bf16(got.cpu().numpy(), want, scale, "gat bf16 width %d" % width)
+
+
+# ------------------------------------------------------------------ host-buffer front end
+
+def test_host_pipeline_matches_direct_calls(g):
+    from paper_2104_03058_b200.host import HostGcnPipeline
+    n, f, ld = 3000, 20, 24
+    jobs = []
+    for seed in range(4):
+        src, dst = gg.powerlaw_graph(n, 30_000, 2.1, None, seed)
+        x = gg.features_f32(n, f, ld=ld, dist="normal", p0=0, p1=1, seed=seed)
+        jobs.append((torch.from_numpy(src).pin_memory(), torch.from_numpy(dst).pin_memory(),
+                     torch.from_numpy(x).pin_memory()))
+    max_e = max(j[0].numel() for j in jobs)
+    pipe = HostGcnPipeline(n, max_e, f, ld, SL, 8)
+    outs = [torch.zeros((n, ld)).pin_memory() for _ in jobs]
+    for i, job in enumerate(jobs):
+        pipe.submit(*job, outs[i], next_job=jobs[i + 1] if i + 1 < len(jobs) else None)
+    pipe.finish()
+    torch.cuda.synchronize()
+    for (h_src, h_dst, h_x), out in zip(jobs, outs):
+        csr = g.build_csr(n, h_src.cuda(), h_dst.cuda(), SL)
+        want = g.aggregate_gcn(csr, h_x.cuda(), f=f, chunk_width=8)
+        assert torch.equal(out[:, :f], want.cpu())
