@@ -1,8 +1,12 @@
 #!/usr/bin/env python
-"""Benchmark of the aggregation hot path: one step = CSR build + chunked GCN aggregation on the
-Reddit-shaped synthetic workload (config 4: 232,965 vertices, ~115M edges + self-loops, F = 602 fp32).
+"""Benchmark of the aggregation hot path.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--chunk-width C]
+One step = gnnfd_build_csr + one chunked aggregation (GCN, GraphSAGE mean or GAT, as the workload
+says) over one synthetic graph.  The default workload is the Reddit-shaped config 4 (232,965
+vertices, ~115M edges + self-loops, F = 602 fp32, GCN); the other configs are available with
+--workload for the results tables and the profiles.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload W] [--chunk-width C]
 
 Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank processes its own graph of the
 same shape (different seed): weak scaling, no data-path collective.  --impl reference times the CPU
@@ -29,22 +33,41 @@ import graphgen as gg  # noqa: E402
 
 METRIC = "aggregated edge-features/sec"
 UNIT = "edge-features/s"
+
+# name -> (factory, default chunk width, description)
 WORKLOADS = {
-    "config4": dict(kind="config4", desc="GCN, 232,965 vertices, ~115M power-law edges + self-loops, F=602 fp32 (ld 608)"),
-    "config4_small": dict(kind="config4", factor=0.25, desc="config 4 recipe at 1/4 of the vertices and 1/16 of the edges"),
+    "config1": (lambda s: gg.config1(s), 16, "GCN, 4,096 vertices, ~40k power-law edges + self-loops, F=16 fp32"),
+    "config2": (lambda s: gg.config2(s), 64, "GraphSAGE mean, 100,000 vertices, avg degree 20 power law, F=128 fp32"),
+    "config3": (lambda s: gg.config3(s), 64,
+                "GAT, 200,000 vertices, avg degree 15 power law + self-loops, 8 heads x 8 dims fp32"),
+    "config4": (lambda s: gg.config4(s), 64,
+                "GCN, 232,965 vertices, ~115M power-law edges + self-loops, F=602 fp32 (ld 608)"),
+    "config4_small": (lambda s: gg.scaled("config4", 0.25, s), 64,
+                      "config 4 recipe at 1/4 of the vertices and 1/16 of the edges"),
+    "config5_f256": (lambda s: gg.config5(s, f=256), 256,
+                     "GCN, RMAT scale 21, 60M edges symmetrised + dedup + self-loops, F=256 bf16"),
+    "config5_f64": (lambda s: gg.config5(s, f=64), 64, "GCN, RMAT scale 21 (as config5_f256), F=64 bf16"),
+    "config5_f32": (lambda s: gg.config5(s, f=32), 32, "GCN, RMAT scale 21 (as config5_f256), F=32 bf16"),
+    "config5_f16": (lambda s: gg.config5(s, f=16), 16, "GCN, RMAT scale 21 (as config5_f256), F=16 bf16"),
+    "config5_f8": (lambda s: gg.config5(s, f=8), 8, "GCN, RMAT scale 21 (as config5_f256), F=8 bf16"),
 }
+KERNEL_OF_MODEL = {"gcn": "gather_aggregate_gcn", "sage": "gather_aggregate_sage", "gat": "gat_aggregate"}
 
 
 def make_workload(name: str, seed: int):
-    spec = WORKLOADS[name]
-    if "factor" in spec:
-        return gg.scaled("config4", spec["factor"], seed)
-    return gg.config4(seed)
+    return WORKLOADS[name][0](seed)
 
 
-def roofline_bytes(n: int, nnz: int, f: int, elem: int, weighted: bool = True) -> int:
-    """CSR indices and weights once, each row pointer once, every gathered feature."""
-    return 4 * (n + 1) + 4 * nnz + (4 * nnz if weighted else 0) + nnz * f * elem
+def roofline_bytes(w, nnz: int) -> int:
+    """Algorithmic bytes of one aggregation launch: every row pointer once, the CSR column indices once,
+    the GCN weights once, every gathered feature (and, for GAT, every gathered score)."""
+    elem = 2 if w.dtype == "bf16" else 4
+    b = 4 * (w.n + 1) + 4 * nnz + nnz * w.f * elem
+    if w.model == "gcn":
+        b += 4 * nnz
+    if w.model == "gat":
+        b += 4 * nnz * w.heads
+    return b
 
 
 def measured_peaks():
@@ -72,13 +95,13 @@ class ClockSampler:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
                  "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.file, stderr=subprocess.DEVNULL)
+            time.sleep(0.3)        # let the sampler come up before the timed region starts
         except OSError:
             self.proc = None
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.15)
         self.proc.terminate()
         self.proc.wait()
         self.file.flush()
@@ -116,12 +139,21 @@ def oracle_sample(w, rows_in_sample: int, seed: int = 0):
 
 
 def oracle_step(w, rows, src, dst, threads: int):
-    """CSR build + GCN aggregation of the sampled rows with the CPU oracle; returns edge-features done."""
+    """CSR build + aggregation of the sampled rows with the CPU oracle; returns edge-features done."""
     import oracle as orc
     row_ptr, col, _ = orc.build_csr(w.n, src, dst, w.flags)
-    orc.aggregate("gcn", row_ptr, col, w.x, w.f, chunk_width=w.f, rows=rows, threads=threads)
+    if w.model == "gat":
+        orc.aggregate_gat(row_ptr, col, w.x, w.a_src, w.a_dst, w.heads, w.dim, w.negative_slope, rows=rows,
+                          threads=threads)
+    else:
+        orc.aggregate(w.model, row_ptr, col, w.x, w.f, chunk_width=w.f, rows=rows, threads=threads)
     deg = np.diff(row_ptr)
     return int(deg[rows].sum()) * w.f
+
+
+def sample_text(w, n_rows: int) -> str:
+    return "CSR build + %s aggregation (F=%d, fp64) of the in-edges of %d sampled destination rows" % (
+        w.model.upper(), w.f, n_rows)
 
 
 def run_reference(args):
@@ -140,13 +172,12 @@ def run_reference(args):
         units += oracle_step(w, rows, src, dst, threads)
     dt = time.perf_counter() - t0
     value = units / dt
-    sample = "CSR build + GCN aggregation (F=%d, fp64) of the in-edges of %d sampled destination rows per step" % (
-        w.f, len(rows))
+    sample = sample_text(w, len(rows)) + " per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "description": WORKLOADS[args.workload]["desc"], "sample": sample},
+        "config": {"workload": args.workload, "description": WORKLOADS[args.workload][2], "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -160,6 +191,8 @@ def run_ours(args):
     import torch.distributed as dist
 
     import paper_2104_03058_b200 as g
+    from paper_2104_03058_b200 import sharding
+    from paper_2104_03058_b200.host import HostPipeline
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -173,10 +206,12 @@ def run_ours(args):
     g.lib()
 
     w = make_workload(args.workload, args.seed + rank)
+    cw = args.chunk_width or WORKLOADS[args.workload][1]
     e = len(w.src)
+    bf16 = w.dtype == "bf16"
     h_src = torch.from_numpy(w.src).pin_memory()
     h_dst = torch.from_numpy(w.dst).pin_memory()
-    h_x = torch.from_numpy(w.x).pin_memory()
+    h_x = (torch.from_numpy(w.x.view(np.int16)).view(torch.bfloat16) if bf16 else torch.from_numpy(w.x)).pin_memory()
     d_src, d_dst, d_x = h_src.to(device), h_dst.to(device), h_x.to(device)
     out = torch.empty((w.n, w.ld), dtype=torch.float32, device=device)
     h_out = torch.empty((w.n, w.ld), dtype=torch.float32).pin_memory()
@@ -184,18 +219,29 @@ def run_ours(args):
     persistent = torch.empty(pb, dtype=torch.uint8, device=device)
     scratch = torch.empty(sb, dtype=torch.uint8, device=device)
     out_view = out[:, :w.f]
-    cw = args.chunk_width
+    gat = w.model == "gat"
+    a_src = torch.from_numpy(w.a_src).to(device) if gat else None
+    a_dst = torch.from_numpy(w.a_dst).to(device) if gat else None
 
     state = {"agg_scratch": None, "csr": None}
+
+    def aggregate(csr, width):
+        if gat:
+            g.aggregate_gat(csr, d_x, a_src, a_dst, w.heads, w.dim, w.negative_slope, chunk_width=width, out=out_view,
+                            scratch=state["agg_scratch"])
+        elif w.model == "sage":
+            g.aggregate_sage(csr, d_x, f=w.f, chunk_width=width, out=out_view, scratch=state["agg_scratch"])
+        else:
+            g.aggregate_gcn(csr, d_x, f=w.f, chunk_width=width, out=out_view, scratch=state["agg_scratch"])
 
     def step():
         if state["csr"] is not None:
             state["csr"].destroy()
         csr = g.build_csr(w.n, d_src, d_dst, w.flags, persistent=persistent, scratch=scratch)
         if state["agg_scratch"] is None:
-            state["agg_scratch"] = torch.empty(max(g.aggregate_workspace_bytes(csr, w.f), 256), dtype=torch.uint8,
-                                               device=device)
-        g.aggregate_gcn(csr, d_x, f=w.f, chunk_width=cw, out=out_view, scratch=state["agg_scratch"])
+            need = g.gat_workspace_bytes(csr, w.heads, w.dim) if gat else g.aggregate_workspace_bytes(csr, w.f)
+            state["agg_scratch"] = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+        aggregate(csr, cw)
         state["csr"] = csr
         return csr
 
@@ -205,7 +251,8 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         csr = step()
     nnz = csr.nnz
     units_per_step = nnz * w.f
@@ -231,8 +278,8 @@ def run_ours(args):
 
     # ---- end to end: pinned host inputs in, result out, every step (the package's host-buffer front end:
     # double-buffered device copies, the next step's inputs and the previous result travel while the kernels run)
-    from paper_2104_03058_b200.host import HostGcnPipeline
-    pipe = HostGcnPipeline(w.n, e, w.f, w.ld, w.flags, cw, device=device)
+    pipe = HostPipeline(w.n, e, w.f, w.ld, w.flags, cw, device=device, feature_dtype=h_x.dtype, model=w.model,
+                        heads=w.heads, dim=w.dim, a_src=a_src, a_dst=a_dst, negative_slope=w.negative_slope)
     job = (h_src, h_dst, h_x)
     pipe.submit(*job, h_out)                         # warm-up job (allocates the aggregation workspace)
     pipe.finish()
@@ -245,53 +292,65 @@ def run_ours(args):
     ev3.record()
     barrier()
     ms_e2e = ev2.elapsed_time(ev3)
-    h2d = h_src.numel() * 4 + h_dst.numel() * 4 + h_x.numel() * 4
+    h2d = sum(t.numel() * t.element_size() for t in job)
     d2h = h_out.numel() * 4
     del pipe
 
-    # ---- aggregation alone (context for the step time), a few calls
+    # ---- aggregation alone (context for the step time), a few calls per chunk width
     agg_ms = {}
+    reps = 3 if units_per_step > 1e9 else 50
     for width in sorted(set(args.sweep + [cw])):
-        g.aggregate_gcn(state["csr"], d_x, f=w.f, chunk_width=width, out=out_view, scratch=state["agg_scratch"])
+        aggregate(state["csr"], width)
         torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
-        for _ in range(3):
-            g.aggregate_gcn(state["csr"], d_x, f=w.f, chunk_width=width, out=out_view, scratch=state["agg_scratch"])
+        for _ in range(reps):
+            aggregate(state["csr"], width)
         a1.record()
         torch.cuda.synchronize()
-        agg_ms[width] = a0.elapsed_time(a1) / 3
+        agg_ms[width] = a0.elapsed_time(a1) / reps
 
-    t = torch.tensor([ms, ms_e2e, float(units_per_step)], dtype=torch.float64, device=device)
-    if world > 1:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms, ms_e2e, total_units = tmax[0].item(), tmax[1].item(), tsum[2].item()
-    else:
-        total_units = float(units_per_step)
+    softmax_ms = None
+    if gat:        # the materialised edge softmax (alpha per CSR slot) on the same graph, timed alone
+        s_src, s_dst = g.gat_scores(d_x, a_src, a_dst, w.heads, w.dim)
+        alpha = torch.empty((nnz, w.heads), dtype=torch.float32, device=device)
+        g.edge_softmax(state["csr"], s_src, s_dst, w.negative_slope, out=alpha)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(reps):
+            g.edge_softmax(state["csr"], s_src, s_dst, w.negative_slope, out=alpha)
+        a1.record()
+        torch.cuda.synchronize()
+        softmax_ms = a0.elapsed_time(a1) / reps
+
+    ms, total_units = sharding.reduce_job_timing(ms, float(units_per_step), device=device)
+    ms_e2e, _ = sharding.reduce_job_timing(ms_e2e, 0.0, device=device)
 
     if rank == 0:
         peak, peak_src = measured_peaks()
-        name = "gather_aggregate_gcn"
+        name = KERNEL_OF_MODEL[w.model]
         k_ms, k_n = kernels.get(name, (0.0, 0))
-        bytes_launch = roofline_bytes(w.n, nnz, w.f, 4)
+        bytes_launch = roofline_bytes(w, nnz)
         achieved = bytes_launch / (k_ms / k_n * 1e-3) / 1e9 if k_n else None
         total_kernel_ms = sum(v[0] for v in kernels.values())
+        x_mb = w.n * w.ld * (2 if bf16 else 4) // 2 ** 20
         result = {
             "metric": METRIC, "value": total_units * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "steps": args.steps, "warmup": warmup, "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "description": WORKLOADS[args.workload]["desc"],
-                       "step": "gnnfd_build_csr + gnnfd_aggregate_gcn", "n": w.n, "input_edges": e, "nnz": nnz,
-                       "f": w.f, "chunk_width": cw, "parallelism": "independent graphs per GPU" if world > 1 else "1 GPU",
-                       "l2": "inputs larger than L2 (x %d MB, col_idx+weights %d MB per sweep; L2 126 MB)"
-                             % (w.n * w.ld * 4 // 2**20, nnz * 8 // 2**20)},
+            "config": {"workload": args.workload, "description": WORKLOADS[args.workload][2],
+                       "step": "gnnfd_build_csr + gnnfd_aggregate_" + w.model, "n": w.n, "input_edges": e, "nnz": nnz,
+                       "f": w.f, "feature_dtype": w.dtype, "chunk_width": cw,
+                       "parallelism": "independent graphs per GPU" if world > 1 else "1 GPU",
+                       "l2": "inputs vs the 126 MB L2: x %d MB, col_idx+weights %d MB per sweep (no flush between steps)"
+                             % (x_mb, nnz * 8 // 2 ** 20)},
             "roofline": {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak if achieved else None, "peak_source": peak_src,
                          "bytes_per_launch": bytes_launch, "kernel_ms": k_ms / k_n if k_n else None,
-                         "frac_of_8TBs_nominal": achieved / 8000.0 if achieved else None, "traffic": None},
+                         "frac_of_8TBs_nominal": achieved / 8000.0 if achieved else None, "traffic": args.traffic_bytes,
+                         "note": "algorithmic bytes charge every gathered feature, most of which L2/L1 serve: "
+                                 "a fraction above 1 means the kernel runs above the HBM roof on cache hits"},
             "e2e": {"value": total_units * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,
@@ -300,9 +359,11 @@ def run_ours(args):
                             "share": v[0] / total_kernel_ms if total_kernel_ms else None}
                         for k, v in sorted(kernels.items(), key=lambda kv: -kv[1][0])},
             "aggregate_only": {str(k): {"ms": v, "edge_features_per_s": units_per_step / (v * 1e-3),
-                                        "roofline_GBs": roofline_bytes(w.n, nnz, w.f, 4) / (v * 1e-3) / 1e9}
+                                        "roofline_GBs": bytes_launch / (v * 1e-3) / 1e9}
                                for k, v in agg_ms.items()},
         }
+        if softmax_ms is not None:
+            result["edge_softmax_only"] = {"ms": softmax_ms, "alpha_GBs_written": nnz * w.heads * 4 / (softmax_ms * 1e-3) / 1e9}
         if world == 1 and not args.no_cpu_baseline:
             import oracle as orc
             threads = orc.max_threads()
@@ -310,10 +371,8 @@ def run_ours(args):
             t0 = time.perf_counter()
             units = oracle_step(w, rows, s_src, s_dst, threads)
             dt = time.perf_counter() - t0
-            result["cpu_baseline"] = {
-                "value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
-                "sample": "CSR build + GCN aggregation (F=%d, fp64) of the in-edges of %d sampled destination rows"
-                          % (w.f, len(rows))}
+            result["cpu_baseline"] = {"value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                      "seconds": dt, "sample": sample_text(w, len(rows))}
         print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
@@ -326,11 +385,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="config4")
-    ap.add_argument("--chunk-width", type=int, default=64)
+    ap.add_argument("--chunk-width", type=int, default=0, help="0 = the workload's default")
     ap.add_argument("--sweep", type=int, nargs="*", default=[], help="extra chunk widths to time (aggregation only)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-rows", type=int, default=16384, help="destination rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture of the current kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -72,7 +72,13 @@ __device__ __forceinline__ void store_elem(void* out, int out_bf16, int64_t idx,
     else __stcs(static_cast<float*>(out) + idx, val);
 }
 
-constexpr int kLoads = 8;      // 16-byte feature loads kept in flight per lane
+#ifndef GNNFD_GATHER_LOADS
+#define GNNFD_GATHER_LOADS 8
+#endif
+#ifndef GNNFD_GATHER_MIN_BLOCKS
+#define GNNFD_GATHER_MIN_BLOCKS 3
+#endif
+constexpr int kLoads = GNNFD_GATHER_LOADS;      // 16-byte feature loads kept in flight per lane
 
 // One row (or hub segment) per S = LPR * EP lanes.  The S lanes fetch the row's indices and weights
 // S at a time with one coalesced load each (R rounds per batch) and hand them to one another by
@@ -231,7 +237,7 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 }
 
 template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED>
-__global__ void __launch_bounds__(kBlock) gather_aggregate(const __grid_constant__ GatherArgs a)
+__global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggregate(const __grid_constant__ GatherArgs a)
 {
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
     const int chunk = (int)(blockIdx.x / per_chunk);

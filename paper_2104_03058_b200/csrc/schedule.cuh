@@ -6,7 +6,10 @@
 
 namespace gnnfd {
 
-constexpr int kBlock = 256;      // threads per block of the gather kernels
+#ifndef GNNFD_GATHER_BLOCK
+#define GNNFD_GATHER_BLOCK 256
+#endif
+constexpr int kBlock = GNNFD_GATHER_BLOCK;      // threads per block of the gather kernels
 constexpr int kUnroll = 8;       // loads kept in flight per lane
 constexpr int kMaxRanges = 5;
 

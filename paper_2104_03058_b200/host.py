@@ -1,6 +1,6 @@
 """Host-buffer front end: graph and features in pinned host memory in, aggregated features out.
 
-``HostGcnPipeline.submit`` runs one job (CSR build + chunked GCN aggregation) whose inputs and output
+``HostPipeline.submit`` runs one job (CSR build + chunked GCN / SAGE / GAT aggregation) whose inputs and output
 live in pinned host memory.  Device buffers are double-buffered and the copies run on their own
 streams, so the host-to-device copy of the next job and the device-to-host copy of the previous
 result overlap the kernels of the current one.  Only torch plumbing (streams, events, copies) lives
@@ -13,10 +13,14 @@ import torch
 from . import binding as g
 
 
-class HostGcnPipeline:
+class HostPipeline:
     def __init__(self, n: int, max_edges: int, f: int, ld: int, flags: int, chunk_width: int, device=None,
-                 feature_dtype=torch.float32, index_dtype=torch.int32, depth: int = 2):
+                 feature_dtype=torch.float32, index_dtype=torch.int32, depth: int = 2, model: str = "gcn",
+                 heads: int = 1, dim: int = 0, a_src=None, a_dst=None, negative_slope: float = 0.2):
+        if model not in ("gcn", "sage", "gat"):
+            raise ValueError(model)
         self.n, self.f, self.ld, self.flags, self.chunk_width = n, f, ld, flags, chunk_width
+        self.model, self.heads, self.dim, self.negative_slope = model, heads, dim, negative_slope
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
         self.depth = depth
         dev = self.device
@@ -28,6 +32,8 @@ class HostGcnPipeline:
         self.persistent = torch.empty(pb, dtype=torch.uint8, device=dev)
         self.scratch = torch.empty(sb, dtype=torch.uint8, device=dev)
         self.agg_scratch = None
+        self.a_src = None if a_src is None else a_src.to(dev)
+        self.a_dst = None if a_dst is None else a_dst.to(dev)
         self.s_in = torch.cuda.Stream(device=dev)
         self.s_out = torch.cuda.Stream(device=dev)
         self.ev_in = [torch.cuda.Event() for _ in range(depth)]        # inputs of slot arrived
@@ -66,10 +72,19 @@ class HostGcnPipeline:
         self.csr = g.build_csr(self.n, self.d_src[slot][:e], self.d_dst[slot][:e], self.flags,
                                persistent=self.persistent, scratch=self.scratch)
         if self.agg_scratch is None:
-            need = max(g.aggregate_workspace_bytes(self.csr, self.f), 256)
-            self.agg_scratch = torch.empty(need, dtype=torch.uint8, device=self.device)
-        g.aggregate_gcn(self.csr, self.d_x[slot], f=self.f, chunk_width=self.chunk_width,
-                        out=self.d_out[slot][:, :self.f], scratch=self.agg_scratch)
+            need = (g.gat_workspace_bytes(self.csr, self.heads, self.dim) if self.model == "gat"
+                    else g.aggregate_workspace_bytes(self.csr, self.f))
+            self.agg_scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+        out = self.d_out[slot][:, :self.f]
+        if self.model == "gat":
+            g.aggregate_gat(self.csr, self.d_x[slot], self.a_src, self.a_dst, self.heads, self.dim,
+                            self.negative_slope, chunk_width=self.chunk_width, out=out, scratch=self.agg_scratch)
+        elif self.model == "sage":
+            g.aggregate_sage(self.csr, self.d_x[slot], f=self.f, chunk_width=self.chunk_width, out=out,
+                             scratch=self.agg_scratch)
+        else:
+            g.aggregate_gcn(self.csr, self.d_x[slot], f=self.f, chunk_width=self.chunk_width, out=out,
+                            scratch=self.agg_scratch)
         self.ev_done[slot].record(cur)
         with torch.cuda.stream(self.s_out):
             self.s_out.wait_event(self.ev_done[slot])
@@ -82,3 +97,6 @@ class HostGcnPipeline:
         cur = torch.cuda.current_stream(self.device)
         cur.wait_stream(self.s_in)
         cur.wait_stream(self.s_out)
+
+
+HostGcnPipeline = HostPipeline
