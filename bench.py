@@ -51,6 +51,30 @@ WORKLOADS = {
     "config5_f16": (lambda s: gg.config5(s, f=16), 16, "GCN, RMAT scale 21 (as config5_f256), F=16 bf16"),
     "config5_f8": (lambda s: gg.config5(s, f=8), 8, "GCN, RMAT scale 21 (as config5_f256), F=8 bf16"),
 }
+# DRAM bytes per launch of the dominant kernel from a one-pass ncu capture of the same launch
+# (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources they were taken with.
+NCU_TRAFFIC = {"config4": {"bytes": 16.81e9, "sources_sha1": "b40528499973b5bbd197fc40e6cb48909235ec2b"}}
+KERNEL_SOURCES = ("paper_2104_03058_b200/csrc/aggregate.cu", "paper_2104_03058_b200/csrc/schedule.cuh")
+# L2-to-crossbar peak that ncu derives on this part (derived__lts__lts2xbar_bytes.sum.peak_sustained), bytes per clock
+L2_PEAK_BYTES_PER_CLK = 11776
+
+
+def kernel_sources_sha1() -> str:
+    import hashlib
+    h = hashlib.sha1()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(workload: str):
+    rec = NCU_TRAFFIC.get(workload)
+    if rec is None or rec["sources_sha1"] != kernel_sources_sha1():
+        return None
+    return rec["bytes"]
+
+
 KERNEL_OF_MODEL = {"gcn": "gather_aggregate_gcn", "sage": "gather_aggregate_sage", "gat": "gat_aggregate"}
 
 
@@ -348,9 +372,16 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak if achieved else None, "peak_source": peak_src,
                          "bytes_per_launch": bytes_launch, "kernel_ms": k_ms / k_n if k_n else None,
-                         "frac_of_8TBs_nominal": achieved / 8000.0 if achieved else None, "traffic": args.traffic_bytes,
+                         "frac_of_8TBs_nominal": achieved / 8000.0 if achieved else None,
+                         "traffic": ncu_traffic(args.workload),
                          "note": "algorithmic bytes charge every gathered feature, most of which L2/L1 serve: "
                                  "a fraction above 1 means the kernel runs above the HBM roof on cache hits"},
+            "l2_roofline": {"what": "gathered bytes all come from L2 on this workload size (ncu: L1 hit rate ~0 at full "
+                                    "size); achieved = algorithmic bytes / kernel time against the L2-to-crossbar peak",
+                            "achieved": achieved, "peak": L2_PEAK_BYTES_PER_CLK * (clocks["sm_max_mhz"] or 1965.0) / 1e3,
+                            "unit": "GB/s",
+                            "frac": achieved / (L2_PEAK_BYTES_PER_CLK * (clocks["sm_max_mhz"] or 1965.0) / 1e3)
+                            if achieved else None},
             "e2e": {"value": total_units * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,
@@ -390,8 +421,6 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-rows", type=int, default=16384, help="destination rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--traffic-bytes", type=float, default=None,
-                    help="DRAM bytes per launch of the dominant kernel from an ncu capture of the current kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -2,6 +2,7 @@
 // duplicate removal, row pointers, degree normalisers, GCN edge weights and the launch schedule
 // (degree bins, hub segments).  Integer work throughout; the only host synchronisation is the
 // final read of the counters.
+#include <cstddef>
 #include <cstring>
 #include <new>
 
@@ -29,11 +30,14 @@ static inline unsigned blocks_for(size_t count, int per_block)
 
 // Candidate i < e: input edge i.  e <= i < 2e (symmetrise): reverse of edge i - e.  Then one
 // self-loop per vertex (value -1).  key = (dst << src_bits) | src; dropped candidates get the
-// destination n, above every valid key, so the sort moves them behind the kept ones.
+// destination n, above every valid key, so the sort moves them behind the kept ones.  When key and
+// value fit one 64-bit word together (vals == nullptr) the word is key << val_bits | (value + 1) and
+// every later kernel reads the key as word >> val_bits.
 template <typename IdT>
 __global__ void __launch_bounds__(kThreads)
 make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, int64_t e, int64_t m, uint32_t flags,
-          int src_bits, u64* __restrict__ keys, int32_t* __restrict__ vals, BuildCounts* __restrict__ counts)
+          int src_bits, int val_bits, u64* __restrict__ keys, int32_t* __restrict__ vals,
+          BuildCounts* __restrict__ counts)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     const u64 invalid = (u64)n << src_bits;
@@ -53,8 +57,13 @@ make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, i
             s = d = i - e - n_rev; val = -1;
             keep = true;
         }
-        __stcs(keys + i, keep ? (((u64)d << src_bits) | (u64)s) : invalid);
-        __stcs(vals + i, val);
+        const u64 key = keep ? (((u64)d << src_bits) | (u64)s) : invalid;
+        if (vals) {
+            __stcs(keys + i, key);
+            __stcs(vals + i, val);
+        } else {
+            __stcs(keys + i, (key << val_bits) | (u64)(uint32_t)(val + 1));   // value travels in the low bits
+        }
     }
     const int kept = __syncthreads_count(keep);
     const int bads = __syncthreads_count(bad);
@@ -86,11 +95,11 @@ radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int mask, in
 
 struct ScatterSmem {
     u64 keys[kSortTile];
-    int32_t vals[kSortTile];
     int32_t warp_count[kSortWarps][kRadix];
     int32_t digit_base[kRadix];     // first slot of each digit inside the sorted tile
     int32_t to_global[kRadix];      // global position of tile slot i holding digit d: to_global[d] + i
     int32_t scan[kSortWarps];
+    int32_t vals[kSortTile];        // last: not allocated when the values travel inside the keys
 };
 
 // exclusive scan of one value per thread over the block; *total receives the block sum
@@ -122,6 +131,7 @@ __device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int
 // count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
 // digit in shared memory and written out run by run, so that consecutive threads store to
 // consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
+template <bool HAS_VALS>
 __global__ void __launch_bounds__(kThreads, 3)
 radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_in, u64* __restrict__ keys_out,
               int32_t* __restrict__ vals_out, int64_t m, int shift, int mask, int64_t n_tiles,
@@ -152,14 +162,12 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
         const int digit = valid ? ((int)(key[r] >> shift) & mask) : kRadix;
         const unsigned peers = __match_any_sync(0xffffffffu, digit);
         const int leader = __ffs(peers) - 1;
+        // the leader of each digit bumps the warp's running count; a warp's shared-memory atomics on one
+        // address complete in program order, so the rounds need no barrier between them
         int32_t before = 0;
-        if (lane == leader && valid) {
-            before = sm.warp_count[warp][digit];
-            sm.warp_count[warp][digit] = before + __popc(peers);
-        }
+        if (lane == leader && valid) before = atomicAdd(&sm.warp_count[warp][digit], __popc(peers));
         before = __shfl_sync(0xffffffffu, before, leader);
         rank[r] = before + __popc(peers & ((1u << lane) - 1u));
-        __syncwarp();
     }
     __syncthreads();
     {
@@ -193,7 +201,7 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
             const int digit = (int)(key[r] >> shift) & mask;
             const int slot = sm.digit_base[digit] + sm.warp_count[warp][digit] + rank[r];
             sm.keys[slot] = key[r];
-            sm.vals[slot] = __ldcs(vals_in + warp_base + r * 32 + lane);
+            if (HAS_VALS) sm.vals[slot] = __ldcs(vals_in + warp_base + r * 32 + lane);
         }
     }
     __syncthreads();
@@ -202,7 +210,7 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
         const u64 k = sm.keys[i];
         const int64_t pos = (int64_t)sm.to_global[(int)(k >> shift) & mask] + i;
         keys_out[pos] = k;
-        vals_out[pos] = sm.vals[i];
+        if (HAS_VALS) vals_out[pos] = sm.vals[i];
     }
 }
 
@@ -210,24 +218,24 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
 
 // flag[i] = 1 for the first of each run of equal keys among the kept candidates
 __global__ void __launch_bounds__(kThreads)
-flag_first_of_run(const u64* __restrict__ keys, int64_t m, const BuildCounts* __restrict__ counts,
+flag_first_of_run(const u64* __restrict__ keys, int64_t m, int val_bits, const BuildCounts* __restrict__ counts,
                   int32_t* __restrict__ flag)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (i >= m) return;
-    flag[i] = (i < counts->n_valid && (i == 0 || keys[i] != keys[i - 1])) ? 1 : 0;
+    flag[i] = (i < counts->n_valid && (i == 0 || (keys[i] >> val_bits) != (keys[i - 1] >> val_bits))) ? 1 : 0;
 }
 
 __global__ void __launch_bounds__(kThreads)
 compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const int32_t* __restrict__ flag,
-               const int32_t* __restrict__ pos, int64_t m, u64* __restrict__ keys_out, int32_t* __restrict__ perm,
-               BuildCounts* __restrict__ counts)
+               const int32_t* __restrict__ pos, int64_t m, int val_bits, u64* __restrict__ keys_out,
+               int32_t* __restrict__ perm, BuildCounts* __restrict__ counts)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (i >= m) return;
     if (flag[i]) {
         keys_out[pos[i]] = keys[i];
-        perm[pos[i]] = vals[i];
+        perm[pos[i]] = vals ? vals[i] : (int32_t)(keys[i] & ((1ull << val_bits) - 1ull)) - 1;
     }
     if (i == m - 1) counts->nnz = pos[i] + flag[i];
 }
@@ -235,8 +243,8 @@ compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, c
 // row_ptr[v] = number of kept keys with dst < v (binary search in the sorted keys).  Without
 // duplicate removal every kept candidate is an entry, which thread 0 records.
 __global__ void __launch_bounds__(kThreads)
-row_pointers(const u64* __restrict__ keys, BuildCounts* __restrict__ counts, int64_t n, int src_bits, int dedup,
-             int32_t* __restrict__ row_ptr)
+row_pointers(const u64* __restrict__ keys, BuildCounts* __restrict__ counts, int64_t n, int src_bits, int val_bits,
+             int dedup, int32_t* __restrict__ row_ptr)
 {
     const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     const int32_t nnz = dedup ? counts->nnz : counts->n_valid;
@@ -246,7 +254,7 @@ row_pointers(const u64* __restrict__ keys, BuildCounts* __restrict__ counts, int
     int32_t lo = 0, hi = nnz;
     while (lo < hi) {
         const int32_t mid = lo + ((hi - lo) >> 1);
-        if (keys[mid] < target) lo = mid + 1; else hi = mid;
+        if ((keys[mid] >> val_bits) < target) lo = mid + 1; else hi = mid;
     }
     row_ptr[v] = lo;
 }
@@ -296,18 +304,19 @@ degrees_and_classes(const int32_t* __restrict__ row_ptr, int64_t n, float* __res
 
 // col_idx, the GCN weight and (unless the duplicate removal already wrote it) perm of every slot
 __global__ void __launch_bounds__(kThreads)
-finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const BuildCounts* __restrict__ counts,
-                 int src_bits, const float* __restrict__ dinv, int32_t* __restrict__ col_idx,
-                 float* __restrict__ edge_w, int32_t* __restrict__ perm, int64_t m)
+finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals, int write_perm,
+                 const BuildCounts* __restrict__ counts, int src_bits, int val_bits, const float* __restrict__ dinv,
+                 int32_t* __restrict__ col_idx, float* __restrict__ edge_w, int32_t* __restrict__ perm, int64_t m)
 {
     const int64_t k = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (k >= m || k >= counts->nnz) return;
-    const u64 key = __ldcs(keys + k);
+    const u64 word = __ldcs(keys + k);
+    const u64 key = word >> val_bits;
     const int32_t s = (int32_t)(key & ((1ull << src_bits) - 1ull));
     const int32_t d = (int32_t)(key >> src_bits);
     __stcs(col_idx + k, s);
     __stcs(edge_w + k, __ldg(dinv + s) * __ldg(dinv + d));
-    if (vals) __stcs(perm + k, __ldcs(vals + k));
+    if (write_perm) __stcs(perm + k, vals ? __ldcs(vals + k) : (int32_t)(word & ((1ull << val_bits) - 1ull)) - 1);
 }
 
 // segments per hub row; entry n_hub (one past the end) is 0 so that the scan yields the total
@@ -353,6 +362,7 @@ struct BuildLayout {
     int64_t hub_cap;       // upper bound on hub rows
     int64_t seg_cap;       // upper bound on hub segments
     int src_bits, key_bits, passes, digit_bits;
+    int val_bits;          // > 0: keys and values share one 64-bit word (key << val_bits | value + 1)
 };
 
 static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
@@ -379,6 +389,9 @@ static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
     L->key_bits = bits + dst_bits;
     L->passes = (L->key_bits + kMaxDigitBits - 1) / kMaxDigitBits;
     L->digit_bits = (L->key_bits + L->passes - 1) / L->passes;
+    int vb = 1;
+    while ((int64_t(1) << vb) < m + 2) ++vb;                  // values -1 .. m-1 stored as 0 .. m
+    L->val_bits = L->key_bits + vb <= 64 ? vb : 0;
     return GNNFD_OK;
 }
 
@@ -490,58 +503,67 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
     int32_t* vals_alt = S.vals_b;
 
     const bool dedup = (flags & GNNFD_CSR_DEDUP) != 0;
+    const int vb = L.val_bits;
+    const bool packed = vb > 0;                     // values ride in the low bits of the keys
+    const size_t scatter_smem = packed ? offsetof(ScatterSmem, vals) : sizeof(ScatterSmem);
+    GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)sizeof(ScatterSmem)));
+    GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)offsetof(ScatterSmem, vals)));
     if (m > 0) {
+        int32_t* key_vals = packed ? nullptr : vals;
         if (itype == GNNFD_I32)
             GNNFD_LAUNCH("make_keys", s, make_keys<int32_t>, blocks_for(m, kThreads), kThreads, 0,
                          static_cast<const int32_t*>(d_src), static_cast<const int32_t*>(d_dst), n, e, m, flags, L.src_bits,
-                         keys, vals, P.counts);
+                         vb, keys, key_vals, P.counts);
         else
             GNNFD_LAUNCH("make_keys", s, make_keys<long long>, blocks_for(m, kThreads), kThreads, 0,
                          static_cast<const long long*>(d_src), static_cast<const long long*>(d_dst), n, e, m, flags,
-                         L.src_bits, keys, vals, P.counts);
-        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)sizeof(ScatterSmem)));
+                         L.src_bits, vb, keys, key_vals, P.counts);
         const int mask = (1 << L.digit_bits) - 1;
         for (int pass = 0; pass < L.passes; ++pass) {
-            const int shift = pass * L.digit_bits;
+            const int shift = pass * L.digit_bits + vb;
             GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.n_tiles, kThreads, 0, keys, m, shift, mask,
                          L.n_tiles, S.hist);
             rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.n_tiles, S.scan_temp, s);
             if (rc) return rc;
-            GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.n_tiles, kThreads, sizeof(ScatterSmem), keys, vals,
-                         keys_alt, vals_alt, m, shift, mask, L.n_tiles, S.hist);
+            if (packed)
+                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<false>, (unsigned)L.n_tiles, kThreads, scatter_smem, keys,
+                             (const int32_t*)nullptr, keys_alt, (int32_t*)nullptr, m, shift, mask, L.n_tiles, S.hist);
+            else
+                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.n_tiles, kThreads, scatter_smem, keys,
+                             (const int32_t*)vals, keys_alt, vals_alt, m, shift, mask, L.n_tiles, S.hist);
             u64* tk = keys; keys = keys_alt; keys_alt = tk;
             int32_t* tv = vals; vals = vals_alt; vals_alt = tv;
         }
         if (dedup) {
-            GNNFD_LAUNCH("flag_first_of_run", s, flag_first_of_run, blocks_for(m, kThreads), kThreads, 0, keys, m,
+            GNNFD_LAUNCH("flag_first_of_run", s, flag_first_of_run, blocks_for(m, kThreads), kThreads, 0, keys, m, vb,
                          P.counts, S.flags);
             int32_t* pos = vals_alt;   // free after the last pass
             rc = exclusive_scan_i32(S.flags, pos, (size_t)m, S.scan_temp, s);
             if (rc) return rc;
-            GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys, vals, S.flags,
-                         pos, m, keys_alt, P.perm, P.counts);
+            GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys,
+                         packed ? (const int32_t*)nullptr : (const int32_t*)vals, S.flags, pos, m, vb, keys_alt, P.perm,
+                         P.counts);
             u64* tk = keys; keys = keys_alt; keys_alt = tk;
         }
     }
     GNNFD_LAUNCH("row_pointers", s, row_pointers, blocks_for((size_t)n + 1, kThreads), kThreads, 0, keys, P.counts, n,
-                 L.src_bits, dedup ? 1 : 0, P.row_ptr);
+                 L.src_bits, vb, dedup ? 1 : 0, P.row_ptr);
     // keys_alt / vals_alt are free from here on: they take the (degree class, row) pairs
     GNNFD_LAUNCH("degrees_and_classes", s, degrees_and_classes, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
                  P.dinv, P.rdeg, keys_alt, vals_alt, P.counts);
     if (m > 0)
         GNNFD_LAUNCH("finalize_entries", s, finalize_entries, blocks_for(m, kThreads), kThreads, 0, keys,
-                     dedup ? (const int32_t*)nullptr : (const int32_t*)vals, P.counts, L.src_bits, P.dinv, P.col_idx,
-                     P.edge_w, P.perm, m);
+                     packed ? (const int32_t*)nullptr : (const int32_t*)vals, dedup ? 0 : 1, P.counts, L.src_bits, vb,
+                     P.dinv, P.col_idx, P.edge_w, P.perm, m);
     // row_order = rows sorted by degree class, ascending row id inside a class: one stable radix pass
     {
-        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)sizeof(ScatterSmem)));
         GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.row_tiles, kThreads, 0, keys_alt, n, 32, kRadix - 1,
                      L.row_tiles, S.hist);
         rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.row_tiles, S.scan_temp, s);
         if (rc) return rc;
-        GNNFD_LAUNCH("radix_scatter", s, radix_scatter, (unsigned)L.row_tiles, kThreads, sizeof(ScatterSmem), keys_alt,
+        GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.row_tiles, kThreads, sizeof(ScatterSmem), keys_alt,
                      vals_alt, reinterpret_cast<u64*>(S.flags), P.row_order, n, 32, kRadix - 1, L.row_tiles, S.hist);
     }
     // the flag buffer is free again: per-hub-row segment counts
