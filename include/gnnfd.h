@@ -136,6 +136,21 @@ int gnnfd_aggregate_sage(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, g
                          void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
                          void* d_scratch, size_t scratch_bytes, void* stream);
 
+/* Choice of the chunk width.  The paper leaves the number of decomposition layers to the user: it
+ * depends on the device's memory capacity and on the dataset (Section II-B; the granularity sweep of
+ * Section III).  gnnfd_default_chunk_candidates fills `candidates` with f (no decomposition) and the
+ * powers of two below f from 256 down to two 16-byte vectors, and returns how many it wrote.
+ * gnnfd_tune_chunk_width runs the aggregation (model 0 = GCN, 1 = SAGE) twice per candidate on the
+ * caller's own graph and features, times the second call with CUDA events on `stream`, and returns the
+ * fastest width in *best_width (its time in *best_ms, may be NULL).  It synchronises the stream;
+ * d_out holds the result for the last candidate tried.  Other arguments as for gnnfd_aggregate_gcn. */
+int gnnfd_default_chunk_candidates(int32_t f, gnnfd_dtype_t xdt, int32_t* candidates, int capacity);
+
+int gnnfd_tune_chunk_width(const gnnfd_csr_t* csr, int model, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt,
+                           void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, const int32_t* candidates,
+                           int n_candidates, void* d_scratch, size_t scratch_bytes, void* stream,
+                           int32_t* best_width, float* best_ms);
+
 /* GCN aggregation without a caller workspace and without any allocation.  (The paper has no
  * counterpart to this entry point; it exists for the library's users.)
  *

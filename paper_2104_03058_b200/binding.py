@@ -55,6 +55,9 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_aggregate_gcn.argtypes = agg
         L.gnnfd_aggregate_sage.argtypes = agg
         L.gnnfd_aggregate_gcn_static.argtypes = [vp, vp, i64, i32, vp, i64, i32, i32, i32, vp]
+        L.gnnfd_default_chunk_candidates.argtypes = [i32, i32, pp(i32), ctypes.c_int]
+        L.gnnfd_tune_chunk_width.argtypes = [vp, ctypes.c_int, vp, i64, i32, vp, i64, i32, i32, pp(i32), ctypes.c_int,
+                                             vp, sz, vp, pp(i32), pp(fl)]
         L.gnnfd_gat_scores.argtypes = [i64, vp, i64, i32, vp, vp, i32, i32, vp, vp, vp]
         L.gnnfd_gat_workspace_bytes.argtypes = [vp, i32, i32, pp(sz)]
         L.gnnfd_aggregate_gat.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32, vp, sz, vp]
@@ -221,6 +224,36 @@ def aggregate_sage(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width:
                    out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None) -> torch.Tensor:
     return _aggregate(lib().gnnfd_aggregate_sage, "gnnfd_aggregate_sage", csr, x, f, chunk_width, out, out_dtype,
                       scratch, stream)
+
+
+def default_chunk_candidates(f: int, dtype=torch.float32) -> list:
+    buf = (ctypes.c_int32 * 16)()
+    k = lib().gnnfd_default_chunk_candidates(f, F32 if dtype == torch.float32 else BF16, buf, 16)
+    if k < 0:
+        raise GnnfdError(k, "gnnfd_default_chunk_candidates")
+    return list(buf[:k])
+
+
+def tune_chunk_width(csr: Csr, x: torch.Tensor, model: str = "gcn", f: int | None = None, candidates=None,
+                     out: torch.Tensor | None = None, scratch=None, stream=None):
+    """gnnfd_tune_chunk_width: times the candidates on this graph and these features; -> (width, ms)."""
+    f = x.shape[1] if f is None else f
+    candidates = default_chunk_candidates(f, x.dtype) if candidates is None else list(candidates)
+    if out is None:
+        out = torch.empty((csr.n, f), dtype=torch.float32, device=x.device)
+    xp, ldx = _matrix(x, f, "x")
+    op, ldo = _matrix(out, f, "out")
+    need = aggregate_workspace_bytes(csr, f)
+    if scratch is None and need:
+        scratch = _alloc_bytes(need, x.device)
+    sp = ctypes.c_void_p(scratch.data_ptr()) if scratch is not None else None
+    sn = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    arr = (ctypes.c_int32 * len(candidates))(*candidates)
+    best, ms = ctypes.c_int32(), ctypes.c_float()
+    _check(lib().gnnfd_tune_chunk_width(csr.handle, {"gcn": 0, "sage": 1}[model], xp, ldx, _dtype_code(x), op, ldo,
+                                        _dtype_code(out), f, arr, len(candidates), sp, sn, _stream_ptr(stream),
+                                        ctypes.byref(best), ctypes.byref(ms)), "gnnfd_tune_chunk_width")
+    return best.value, ms.value
 
 
 def aggregate_gcn_static(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width: int | None = None,

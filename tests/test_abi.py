@@ -45,3 +45,13 @@ def test_header_constants_match_binding():
     assert int(re.search(r"#define GNNFD_HUB_SEGMENT (\d+)", text).group(1)) == g.HUB_SEGMENT
     for name, val in (("ADD_SELF_LOOPS", 1), ("DEDUP", 2), ("SYMMETRIZE", 4)):
         assert int(re.search(r"GNNFD_CSR_%s = (\d+)" % name, text).group(1)) == val == getattr(g, "CSR_" + name)
+
+
+def test_default_chunk_candidates_are_host_only():
+    import torch
+
+    import paper_2104_03058_b200 as g
+    assert g.default_chunk_candidates(602) == [602, 256, 128, 64, 32, 16, 8]
+    assert g.default_chunk_candidates(64) == [64, 32, 16, 8]
+    assert g.default_chunk_candidates(8, torch.bfloat16) == [8]
+    assert g.default_chunk_candidates(256, torch.bfloat16) == [256, 128, 64, 32, 16]

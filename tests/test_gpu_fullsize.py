@@ -61,3 +61,12 @@ def test_config4_closed_forms_on_every_row(big):
     c = torch.full((w.n, f), 3.25, device="cuda")
     got = g.aggregate_sage(csr, c, f=f, chunk_width=8).cpu().numpy()
     np.testing.assert_allclose(got, 3.25, rtol=2e-5)
+
+
+def test_config4_tuner_prefers_a_decomposed_sweep(big):
+    g, w, csr, _ = big
+    xd = torch.from_numpy(w.x).cuda()
+    out = torch.empty((w.n, w.ld), device="cuda")
+    width, ms = g.tune_chunk_width(csr, xd, "gcn", f=w.f, candidates=[602, 128, 64, 32], out=out[:, :w.f])
+    # the slice gathered per sweep must fit L2: the undecomposed sweep (561 MB) and very narrow chunks lose
+    assert width in (64, 128) and 5.0 < ms < 60.0

@@ -348,3 +348,20 @@ def test_host_pipeline_matches_direct_calls(g):
         csr = g.build_csr(n, h_src.cuda(), h_dst.cuda(), SL)
         want = g.aggregate_gcn(csr, h_x.cuda(), f=f, chunk_width=8)
         assert torch.equal(out[:, :f], want.cpu())
+
+
+def test_chunk_width_tuner_picks_a_candidate_and_leaves_a_valid_result(g):
+    w = gg.scaled("config4", 0.05)
+    row_ptr, col, _ = orc.build_csr(w.n, w.src, w.dst, w.flags)
+    csr = g.build_csr(w.n, dev(w.src), dev(w.dst), w.flags)
+    xd = dev(w.x)
+    out = torch.empty((w.n, w.f), device="cuda")
+    cands = g.default_chunk_candidates(w.f)
+    width, ms = g.tune_chunk_width(csr, xd, "gcn", f=w.f, candidates=cands, out=out)
+    assert width in cands and ms > 0
+    want, scale = orc.aggregate("gcn", row_ptr, col, w.x, w.f, threads=orc.max_threads())
+    assert_close_f32(out.cpu().numpy(), want, scale, "tuner leaves the last candidate's result")
+    width_sage, _ = g.tune_chunk_width(csr, xd, "sage", f=w.f, candidates=[64, 602])
+    assert width_sage in (64, 602)
+    with pytest.raises(g.GnnfdError):
+        g.tune_chunk_width(csr, xd, "gcn", f=w.f, candidates=[0])
