@@ -13,8 +13,10 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "oracle.cpp")
-_LIB = os.path.join(_HERE, "liboracle.so")
+# The two overrides exist for the mutation test, which builds deliberately wrong copies of the source
+# elsewhere and checks that the pins reject them.
+_SRC = os.environ.get("GNNFD_ORACLE_SOURCE", os.path.join(_HERE, "oracle.cpp"))
+_LIB = os.environ.get("GNNFD_ORACLE_LIB", os.path.join(_HERE, "liboracle.so"))
 _lib = None
 
 ADD_SELF_LOOPS, DEDUP, SYMMETRIZE = 1, 2, 4
