@@ -131,8 +131,11 @@ __device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int
 // count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
 // digit in shared memory and written out run by run, so that consecutive threads store to
 // consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
+#ifndef GNNFD_SCATTER_MIN_BLOCKS
+#define GNNFD_SCATTER_MIN_BLOCKS 3
+#endif
 template <bool HAS_VALS>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, GNNFD_SCATTER_MIN_BLOCKS)
 radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_in, u64* __restrict__ keys_out,
               int32_t* __restrict__ vals_out, int64_t m, int shift, int mask, int64_t n_tiles,
               const int32_t* __restrict__ tile_offset)
