@@ -5,8 +5,8 @@
 // thread owns head t % heads and every (S / heads)-th slot, so consecutive threads write
 // consecutive addresses of alpha; otherwise the heads are taken one at a time.  S grows with the
 // degree class of the row (the rows come sorted by degree, so a warp's rows have similar lengths).
-// A hub row is shared by a whole thread-block cluster: the per-head maxima and sums of the member
-// blocks are exchanged through distributed shared memory.
+// Rows of the top degree bin get a block each and hub rows a whole thread-block cluster: the per-head
+// maxima and sums of the member blocks are exchanged through distributed shared memory.
 #include <cooperative_groups.h>
 #include <math_constants.h>
 
@@ -17,9 +17,9 @@ namespace cg = cooperative_groups;
 namespace gnnfd {
 
 constexpr int kRowBlock = 256;          // threads per block, ordinary rows
-constexpr int kHubBlock = 512;          // threads per block, hub rows
+constexpr int kBigBlock = 256;          // threads per block, rows of 129 .. GNNFD_HUB_DEGREE entries (one block each)
+constexpr int kHubBlock = 1024;         // threads per block, hub rows
 constexpr int kHubCluster = 8;          // blocks per hub row
-constexpr int kHubThreads = kHubBlock * kHubCluster;
 
 __device__ __forceinline__ float leaky_relu(float x, float slope) { return x >= 0.f ? x : slope * x; }
 
@@ -38,19 +38,22 @@ __device__ __forceinline__ float logit(const RowView& r, int32_t k, int h, float
     return leaky_relu(__ldg(r.s_src + (int64_t)__ldg(r.col_idx + k) * r.heads + h) + sd, r.slope);
 }
 
-// Running maximum and denominator over slots first, first + step, ... (four logits in flight).
+// Running maximum and denominator over slots first, first + step, ... (kInFlight logits in flight).
+constexpr int kInFlight = 8;
 __device__ __forceinline__ void online_max_sum(const RowView& r, int32_t first, int step, int h, float sd, float* m_out,
                                                float* l_out)
 {
     float m = -CUDART_INF_F, l = 0.f;
-    for (int32_t k = first; k < r.e; k += 4 * step) {
-        float t[4];
+    for (int32_t k = first; k < r.e; k += kInFlight * step) {
+        float t[kInFlight];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : -CUDART_INF_F;
-        const float mx = fmaxf(fmaxf(m, fmaxf(t[0], t[1])), fmaxf(t[2], t[3]));     // t[0] is valid, so mx is finite
+        for (int i = 0; i < kInFlight; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : -CUDART_INF_F;
+        float mx = m;                                                               // t[0] is valid, so mx ends finite
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) mx = fmaxf(mx, t[i]);
         l *= expf(m - mx);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) l += expf(t[i] - mx);                           // exp(-inf) = 0 for the missing ones
+        for (int i = 0; i < kInFlight; ++i) l += expf(t[i] - mx);                   // exp(-inf) = 0 for the missing ones
         m = mx;
     }
     *m_out = m;
@@ -59,12 +62,12 @@ __device__ __forceinline__ void online_max_sum(const RowView& r, int32_t first, 
 
 __device__ __forceinline__ void write_alpha(const RowView& r, int32_t first, int step, int h, float sd, float m, float inv)
 {
-    for (int32_t k = first; k < r.e; k += 4 * step) {
-        float t[4];
+    for (int32_t k = first; k < r.e; k += kInFlight * step) {
+        float t[kInFlight];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : 0.f;
+        for (int i = 0; i < kInFlight; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < kInFlight; ++i)
             if (k + i * step < r.e) __stcs(r.alpha + (int64_t)(k + i * step) * r.heads + h, expf(t[i] - m) * inv);
     }
 }
@@ -86,8 +89,36 @@ edge_softmax_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict
     for (int h0 = 0; h0 < heads; h0 += hh) {
         const int h = h0 + sl % hh;
         const float sd = active ? s_dst[(int64_t)row * heads + h] : 0.f;
+        const int32_t first = r.b + sl / hh;
+        if (__all_sync(0xffffffffu, r.e - r.b <= kInFlight * step)) {
+            // every row of this warp fits one round: the logits stay in registers between the two phases
+            float t[kInFlight];
+            float m = -CUDART_INF_F;
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i) {
+                t[i] = first + i * step < r.e ? logit(r, first + i * step, h, sd) : -CUDART_INF_F;
+                m = fmaxf(m, t[i]);
+            }
+#pragma unroll
+            for (int o = S / 2; o >= 1; o >>= 1)
+                if (o >= hh) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            float l = 0.f;
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i) {
+                t[i] = first + i * step < r.e ? expf(t[i] - m) : 0.f;
+                l += t[i];
+            }
+#pragma unroll
+            for (int o = S / 2; o >= 1; o >>= 1)
+                if (o >= hh) l += __shfl_xor_sync(0xffffffffu, l, o);
+            const float inv = 1.f / l;
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i)
+                if (first + i * step < r.e) __stcs(alpha + (int64_t)(first + i * step) * heads + h, t[i] * inv);
+            continue;
+        }
         float m, l;
-        online_max_sum(r, r.b + sl / hh, step, h, sd, &m, &l);
+        online_max_sum(r, first, step, h, sd, &m, &l);
         float mall = m;
 #pragma unroll
         for (int o = S / 2; o >= 1; o >>= 1)
@@ -96,15 +127,15 @@ edge_softmax_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict
 #pragma unroll
         for (int o = S / 2; o >= 1; o >>= 1)
             if (o >= hh) l += __shfl_xor_sync(0xffffffffu, l, o);
-        write_alpha(r, r.b + sl / hh, step, h, sd, mall, 1.f / l);
+        write_alpha(r, first, step, h, sd, mall, 1.f / l);
     }
 }
 
-// ---- hub rows: one cluster of kHubCluster blocks per row
+// ---- long rows: one block, hub rows: one cluster of blocks per row
 
 // Combines one value per thread over all threads of the cluster that own the same head (threads with
 // equal t % hh; hh divides 32).  `mine` is this block's exchange buffer of 32 floats.
-template <bool IS_MAX>
+template <bool IS_MAX, int THREADS, int CLUSTER>
 __device__ __forceinline__ float cluster_combine(float v, int hh, float* warp_buf, float* mine, cg::cluster_group& cluster)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -114,21 +145,21 @@ __device__ __forceinline__ float cluster_combine(float v, int hh, float* warp_bu
             const float other = __shfl_xor_sync(0xffffffffu, v, o);
             v = IS_MAX ? fmaxf(v, other) : v + other;
         }
+    __syncthreads();                                  // the previous combine's readers are done
     warp_buf[warp * 32 + lane] = v;
     __syncthreads();
-    if (warp == 0) {
-        float acc = warp_buf[lane];
+    float acc = warp_buf[lane];
 #pragma unroll
-        for (int w = 1; w < kHubBlock / 32; ++w) {
-            const float other = warp_buf[w * 32 + lane];
-            acc = IS_MAX ? fmaxf(acc, other) : acc + other;
-        }
-        mine[lane] = acc;
+    for (int w = 1; w < THREADS / 32; ++w) {
+        const float other = warp_buf[w * 32 + lane];
+        acc = IS_MAX ? fmaxf(acc, other) : acc + other;
     }
+    if (CLUSTER == 1) return acc;
+    if (warp == 0) mine[lane] = acc;
     cluster.sync();                                   // every block's `mine` is complete
-    float acc = IS_MAX ? -CUDART_INF_F : 0.f;
+    acc = IS_MAX ? -CUDART_INF_F : 0.f;
 #pragma unroll
-    for (int rk = 0; rk < kHubCluster; ++rk) {
+    for (int rk = 0; rk < CLUSTER; ++rk) {
         const float other = cluster.map_shared_rank(mine, rk)[lane];
         acc = IS_MAX ? fmaxf(acc, other) : acc + other;
     }
@@ -136,26 +167,31 @@ __device__ __forceinline__ float cluster_combine(float v, int hh, float* warp_bu
     return acc;
 }
 
-__global__ void __cluster_dims__(kHubCluster, 1, 1) __launch_bounds__(kHubBlock)
-edge_softmax_hubs(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                  const int32_t* __restrict__ hub_rows, const float* __restrict__ s_src, const float* __restrict__ s_dst,
-                  int heads, int hh, float slope, float* __restrict__ alpha)
+template <int THREADS, int CLUSTER>
+__global__ void __cluster_dims__(CLUSTER, 1, 1) __launch_bounds__(THREADS)
+edge_softmax_big(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                 const int32_t* __restrict__ rows, const float* __restrict__ s_src, const float* __restrict__ s_dst,
+                 int heads, int hh, float slope, int32_t min_len, int32_t max_len, float* __restrict__ alpha)
 {
-    __shared__ float warp_buf[kHubBlock];
+    __shared__ float warp_buf[THREADS];
     __shared__ float mine[32];
     cg::cluster_group cluster = cg::this_cluster();
-    const int32_t row = hub_rows[blockIdx.x / kHubCluster];
-    const int t = (int)cluster.block_rank() * kHubBlock + threadIdx.x;
+    const int32_t row = rows[blockIdx.x / CLUSTER];
+    {   // rows outside [min_len, max_len] belong to another launch; the whole cluster leaves together
+        const int32_t len = row_ptr[row + 1] - row_ptr[row];
+        if (len < min_len || len > max_len) return;
+    }
+    const int t = (CLUSTER == 1 ? 0 : (int)cluster.block_rank() * THREADS) + threadIdx.x;
     RowView r{col_idx, s_src, alpha, row_ptr[row], row_ptr[row + 1], heads, slope};
-    const int step = kHubThreads / hh;
+    const int step = THREADS * CLUSTER / hh;
     for (int h0 = 0; h0 < heads; h0 += hh) {
         const int h = h0 + t % hh;
         const float sd = s_dst[(int64_t)row * heads + h];
         float m, l;
         online_max_sum(r, r.b + t / hh, step, h, sd, &m, &l);
-        const float mall = cluster_combine<true>(m, hh, warp_buf, mine, cluster);
+        const float mall = cluster_combine<true, THREADS, CLUSTER>(m, hh, warp_buf, mine, cluster);
         l = m == -CUDART_INF_F ? 0.f : l * expf(m - mall);
-        l = cluster_combine<false>(l, hh, warp_buf, mine, cluster);
+        l = cluster_combine<false, THREADS, CLUSTER>(l, hh, warp_buf, mine, cluster);
         write_alpha(r, r.b + t / hh, step, h, sd, mall, 1.f / l);
     }
 }
@@ -184,8 +220,8 @@ extern "C" int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, 
     if (!csr || !d_s_src || !d_s_dst || !d_alpha || heads <= 0) return GNNFD_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int hh = (heads <= 32 && (heads & (heads - 1)) == 0) ? heads : 1;   // heads handled together
-    static const int slots_in_parallel[4] = {2, 8, 32, 32};                   // per degree class of the row
-    for (int bin = 0; bin < 4; ++bin) {
+    static const int slots_in_parallel[3] = {2, 8, 32};                       // per degree bin of the row
+    for (int bin = 0; bin < 3; ++bin) {
         const int64_t rows = csr->bin_count[bin];
         if (rows == 0) continue;
         int lanes = hh * slots_in_parallel[bin];
@@ -195,11 +231,15 @@ extern "C" int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, 
         GNNFD_LAUNCH("edge_softmax_rows", s, pick_rows(lanes), grid, kRowBlock, 0, csr->row_ptr, csr->col_idx,
                      csr->row_order + csr->bin_start[bin], rows, d_s_src, d_s_dst, heads, hh, negative_slope, d_alpha);
     }
+    if (csr->bin_count[3] > 0)
+        GNNFD_LAUNCH("edge_softmax_long_rows", s, (edge_softmax_big<kBigBlock, 1>), (unsigned)csr->bin_count[3], kBigBlock, 0,
+                     csr->row_ptr, csr->col_idx, csr->row_order + csr->bin_start[3], d_s_src, d_s_dst, heads, hh,
+                     negative_slope, 0, 0x7fffffff, d_alpha);
     const int64_t n_hub = csr->bin_count[4];
     if (n_hub > 0)
-        GNNFD_LAUNCH("edge_softmax_hubs", s, edge_softmax_hubs, (unsigned)(n_hub * kHubCluster), kHubBlock, 0, csr->row_ptr,
-                     csr->col_idx, csr->row_order + csr->bin_start[4], d_s_src, d_s_dst, heads, hh, negative_slope,
-                     d_alpha);
+        GNNFD_LAUNCH("edge_softmax_hubs", s, (edge_softmax_big<kHubBlock, kHubCluster>), (unsigned)(n_hub * kHubCluster),
+                     kHubBlock, 0, csr->row_ptr, csr->col_idx, csr->row_order + csr->bin_start[4], d_s_src, d_s_dst, heads,
+                     hh, negative_slope, 0, 0x7fffffff, d_alpha);
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
 }

@@ -296,27 +296,48 @@ __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ 
     }
 }
 
-// out[row, j] = sum_s partial[s, j] e^(m_s - M) / sum_s l_s e^(m_s - M), segments in ascending order
+// out[row, j] = sum_s partial[s, j] e^(m_s - M) / sum_s l_s e^(m_s - M) over the segments s of a hub row.
+// A block covers kReduceCols columns of one row; kReduceWays threads per column walk interleaved
+// segments and their results are combined in a fixed order through shared memory.
+constexpr int kReduceCols = 64;
+constexpr int kReduceWays = kBlock / kReduceCols;
+
 __global__ void __launch_bounds__(kBlock)
 gat_hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict__ hub_seg_ptr,
                const float* __restrict__ partial, const float* __restrict__ partial_ml, int64_t hub_begin, int32_t n_hub,
                int32_t f, int32_t fpad, int32_t heads, int32_t dim, void* __restrict__ out, int64_t ldo, int out_bf16)
 {
+    __shared__ float s_max[kReduceWays][kReduceCols], s_num[kReduceWays][kReduceCols], s_den[kReduceWays][kReduceCols];
     const int i = blockIdx.x;
-    const int j = blockIdx.y * kBlock + threadIdx.x;
-    if (i >= n_hub || j >= f) return;
-    const int h = j / dim;
+    const int c = threadIdx.x % kReduceCols, q = threadIdx.x / kReduceCols;
+    const int j = blockIdx.y * kReduceCols + c;
+    const bool ok = j < f;
+    const int h = ok ? j / dim : 0;
     const int32_t row = row_order[hub_begin + i];
     const int32_t s0 = hub_seg_ptr[i], s1 = hub_seg_ptr[i + 1];
     float mx = -CUDART_INF_F;
-    for (int32_t s = s0; s < s1; ++s) mx = fmaxf(mx, partial_ml[((int64_t)s * heads + h) * 2]);
+    if (ok)
+        for (int32_t s = s0 + q; s < s1; s += kReduceWays) mx = fmaxf(mx, partial_ml[((int64_t)s * heads + h) * 2]);
+    s_max[q][c] = mx;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kReduceWays; ++w) mx = fmaxf(mx, s_max[w][c]);
     float num = 0.f, den = 0.f;
-    for (int32_t s = s0; s < s1; ++s) {
-        const float* ml = partial_ml + ((int64_t)s * heads + h) * 2;
-        const float w = merge_scale(ml[0], mx);
-        den = fmaf(ml[1], w, den);
-        num = fmaf(partial[(int64_t)s * fpad + j], w, num);
-    }
+    if (ok)
+        for (int32_t s = s0 + q; s < s1; s += kReduceWays) {
+            const float* ml = partial_ml + ((int64_t)s * heads + h) * 2;
+            const float w = merge_scale(ml[0], mx);
+            den = fmaf(ml[1], w, den);
+            num = fmaf(partial[(int64_t)s * fpad + j], w, num);
+        }
+    s_num[q][c] = num;
+    s_den[q][c] = den;
+    __syncthreads();
+    if (q != 0 || !ok) return;
+    num = 0.f;
+    den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kReduceWays; ++w) { num += s_num[w][c]; den += s_den[w][c]; }
     store_out(out, out_bf16, (int64_t)row * ldo + j, den > 0.f ? num / den : 0.f);
 }
 
@@ -454,7 +475,7 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     }
     const int64_t n_hub = csr->bin_count[4];
     if (n_hub > 0) {
-        dim3 gr((unsigned)n_hub, (unsigned)((f + kBlock - 1) / kBlock));
+        dim3 gr((unsigned)n_hub, (unsigned)((f + kReduceCols - 1) / kReduceCols));
         GNNFD_LAUNCH("gat_hub_reduce", s, gat_hub_reduce, gr, kBlock, 0, csr->row_order, csr->hub_seg_ptr, g.partial,
                      g.partial_ml, csr->bin_start[4], (int32_t)n_hub, f, a.fpad, heads, dim, d_out, ldo, a.out_bf16);
     }
