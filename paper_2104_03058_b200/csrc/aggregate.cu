@@ -7,7 +7,7 @@
 // x, which is what keeps the gathered working set small enough for L2.  Inside a sweep the rows come
 // grouped by degree class.  A row is owned by S = LPR * EP lanes: LPR lanes cover the chunk's columns
 // with one or two 16-byte vectors each, and EP groups of LPR lanes walk interleaved entries of the
-// row, each keeping 8 loads in flight.  The EP partial sums are combined by a fixed shuffle tree, hub rows
+// row, each keeping 8 loads in flight; column indices and edge weights are staged per warp in shared memory.  The EP partial sums are combined by a fixed shuffle tree, hub rows
 // (degree > GNNFD_HUB_DEGREE) by per-segment partial sums that a second kernel adds in ascending
 // segment order: no atomics, bit-identical from run to run.
 #include <cuda_bf16.h>
@@ -80,15 +80,19 @@ __device__ __forceinline__ void store_elem(void* out, int out_bf16, int64_t idx,
 #endif
 constexpr int kLoads = GNNFD_GATHER_LOADS;      // 16-byte feature loads kept in flight per lane
 
+constexpr int kStageSlots = kLoads * 32;      // column indices (and weights) a warp stages per batch, at most
+
 // One row (or hub segment) per S = LPR * EP lanes.  The S lanes fetch the row's indices and weights
-// S at a time with one coalesced load each (R rounds per batch) and hand them to one another by
-// shuffle: in step s of a batch, group g works on entry r*S + t*EP + g (r = s / LPR, t = s % LPR),
-// which lane t*EP + g of the segment holds in its r-th register.  A lane covers VPL vectors of the
+// S at a time with one coalesced streaming load each (R rounds per batch) and stage them in the
+// warp's shared-memory buffer (double-buffered; the next batch is already in registers, on its way
+// from HBM, while this one is consumed).  In step s of a batch, group g works on entry
+// r*S + t*EP + g (r = s / LPR, t = s % LPR), read back as a broadcast.  A lane covers VPL vectors of the
 // chunk (columns c + q*LPR, q < VPL, in vector units) so that the index traffic, the address
 // arithmetic and the shuffles are paid once per VPL * 16 gathered bytes.
 template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, int EP>
 __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0,
-                                            int chunk_end)
+                                            int chunk_end, int32_t (*stage_col)[kBlock / 32][kStageSlots],
+                                            float (*stage_w)[kBlock / 32][kStageSlots])
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
@@ -102,6 +106,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     const int sl = tid % S;
     const int g = sl / LPR;
     const int c = sl % LPR;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int seg = lane - sl;                   // first lane of this row's segment inside the warp
     const bool active = slot < rg.item_count;
 
     int jq[VPL];
@@ -159,6 +165,13 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
             wnext[r] = (WEIGHTED && ok) ? __ldcs(a.edge_w + kk) : 0.f;
         }
         const bool full = __all_sync(kFull, kb + EPB <= e);
+        const int buf = ib & 1;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            stage_col[buf][warp][r * 32 + lane] = ucur[r];
+            if (WEIGHTED) stage_w[buf][warp][r * 32 + lane] = wcur[r];
+        }
+        __syncwarp();
 #pragma unroll
         for (int s0 = 0; s0 < SPB; s0 += UB) {
             Vec<T, VECN> v[UB][VPL];
@@ -167,8 +180,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
                     const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
-                    if (WEIGHTED) wv[i] = __shfl_sync(kFull, wcur[r], t * EP + g, S);
+                    const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
+                    if (WEIGHTED) wv[i] = stage_w[buf][warp][r * 32 + seg + t * EP + g];
                     const size_t off = (size_t)(uint32_t)u * ld;
 #pragma unroll
                     for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
@@ -177,8 +190,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
                     const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
-                    if (WEIGHTED) wv[i] = __shfl_sync(kFull, wcur[r], t * EP + g, S);
+                    const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
+                    if (WEIGHTED) wv[i] = stage_w[buf][warp][r * 32 + seg + t * EP + g];
                     const size_t off = (size_t)(uint32_t)max(u, 0) * ld;
 #pragma unroll
                     for (int q = 0; q < VPL; ++q) {
@@ -239,6 +252,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED>
 __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggregate(const __grid_constant__ GatherArgs a)
 {
+    __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
+    __shared__ float stage_w[2][kBlock / 32][kStageSlots];
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
     const int chunk = (int)(blockIdx.x / per_chunk);
     const int rem = (int)(blockIdx.x % per_chunk);
@@ -255,12 +270,12 @@ __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggreg
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end); break;
-        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end); break;
-        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end); break;
-        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end); break;
-        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end); break;
-        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end); break;
+        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
     }
 }
 

@@ -104,11 +104,14 @@ gat_scores(const T* __restrict__ z, int64_t ldz, const float* __restrict__ a_src
 
 constexpr int kLoads = 8;      // 16-byte feature loads kept in flight per lane
 
+constexpr int kStageSlots = kLoads * 32;      // column indices a warp stages per batch, at most
+
 // One row (or hub segment) per S = LPR * EP lanes, same batching as the GCN / SAGE gather: the S lanes
-// fetch S column indices per round with one coalesced load and pass them on by shuffle.  A lane
+// fetch S column indices per round with one coalesced load and stage them in shared memory.  A lane
 // covers VPL adjacent vectors, all inside one head, so it needs one logit per entry.
 template <typename T, int VECN, int LPR, int VPL, int EP>
-__device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int block_in_range, int col0, int chunk_end)
+__device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int block_in_range, int col0, int chunk_end,
+                                         int32_t (*stage_col)[kBlock / 32][kStageSlots])
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
@@ -123,6 +126,8 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
     const int g = sl / LPR;
     const int c = sl % LPR;
     const int j0 = col0 + c * (VPL * VECN);
+    const int warp = tid >> 5, lane = tid & 31;
+    const int seg = lane - sl;                   // first lane of this row's segment inside the warp
     const bool active = slot < rg.item_count;
     const bool lane_ok = j0 < chunk_end;
     const int h = (lane_ok ? j0 : col0) / a.dim;
@@ -175,6 +180,10 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
             const int32_t kk = kb + EPB + r * S + sl;
             unext[r] = kk < e ? __ldcs(a.col_idx + kk) : -1;
         }
+        const int buf = ib & 1;
+#pragma unroll
+        for (int r = 0; r < R; ++r) stage_col[buf][warp][r * 32 + lane] = ucur[r];
+        __syncwarp();
 #pragma unroll
         for (int s0 = 0; s0 < SPB; s0 += UB) {
             ZVec<T, VECN> v[UB][VPL];
@@ -183,7 +192,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
 #pragma unroll
             for (int i = 0; i < UB; ++i) {
                 const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                const int32_t u = __shfl_sync(kFull, ucur[r], t * EP + g, S);
+                const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
                 valid[i] = u >= 0;
                 const uint32_t uu = (uint32_t)max(u, 0);
                 lg[i] = valid[i] ? __ldg(ssrc + (size_t)uu * heads) : 0.f;
@@ -271,6 +280,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
 template <typename T, int VECN, int LPR, int VPL>
 __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ GatArgs a)
 {
+    __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
     const int chunk = (int)(blockIdx.x / per_chunk);
     const int rem = (int)(blockIdx.x % per_chunk);
@@ -287,12 +297,12 @@ __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ 
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gat_rows<T, VECN, LPR, VPL, 1>(a, rg, bir, col0, chunk_end); break;
-        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, VPL, 2>(a, rg, bir, col0, chunk_end); break;
-        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, VPL, 4>(a, rg, bir, col0, chunk_end); break;
-        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, VPL, 8>(a, rg, bir, col0, chunk_end); break;
-        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, VPL, 16>(a, rg, bir, col0, chunk_end); break;
-        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, VPL, 32>(a, rg, bir, col0, chunk_end); break;
+        case 0: gat_rows<T, VECN, LPR, VPL, 1>(a, rg, bir, col0, chunk_end, stage_col); break;
+        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, VPL, 2>(a, rg, bir, col0, chunk_end, stage_col); break;
+        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, VPL, 4>(a, rg, bir, col0, chunk_end, stage_col); break;
+        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, VPL, 8>(a, rg, bir, col0, chunk_end, stage_col); break;
+        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, VPL, 16>(a, rg, bir, col0, chunk_end, stage_col); break;
+        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, VPL, 32>(a, rg, bir, col0, chunk_end, stage_col); break;
     }
 }
 
