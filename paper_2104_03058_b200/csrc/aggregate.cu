@@ -166,12 +166,14 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         }
         const bool full = __all_sync(kFull, kb + EPB <= e);
         const int buf = ib & 1;
+        if (LPR > 1) {      // with one lane per row every lane consumes exactly the entries it fetched
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            stage_col[buf][warp][r * 32 + lane] = ucur[r];
-            if (WEIGHTED) stage_w[buf][warp][r * 32 + lane] = wcur[r];
+            for (int r = 0; r < R; ++r) {
+                stage_col[buf][warp][r * 32 + lane] = ucur[r];
+                if (WEIGHTED) stage_w[buf][warp][r * 32 + lane] = wcur[r];
+            }
+            __syncwarp();
         }
-        __syncwarp();
 #pragma unroll
         for (int s0 = 0; s0 < SPB; s0 += UB) {
             Vec<T, VECN> v[UB][VPL];
@@ -180,8 +182,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
                     const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
-                    if (WEIGHTED) wv[i] = stage_w[buf][warp][r * 32 + seg + t * EP + g];
+                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
+                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)u * ld;
 #pragma unroll
                     for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
@@ -190,8 +192,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
                     const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
-                    if (WEIGHTED) wv[i] = stage_w[buf][warp][r * 32 + seg + t * EP + g];
+                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
+                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)max(u, 0) * ld;
 #pragma unroll
                     for (int q = 0; q < VPL; ++q) {
