@@ -10,9 +10,8 @@
 // row, each keeping 8 loads in flight; column indices and edge weights are staged per warp in shared memory.  The EP partial sums are combined by a fixed shuffle tree, hub rows
 // (degree > GNNFD_HUB_DEGREE) by per-segment partial sums that a second kernel adds in ascending
 // segment order: no atomics, bit-identical from run to run.
-#include <cuda_bf16.h>
-
 #include "schedule.cuh"
+#include "vec.cuh"
 
 namespace gnnfd {
 
@@ -32,45 +31,6 @@ struct GatherArgs {
     int32_t n_ranges;
     Range range[kMaxRanges];
 };
-
-// ---- per-lane vectors: VECN elements of T, widened to fp32
-
-template <typename T, int VECN> struct Vec;
-
-template <> struct Vec<float, 4> {
-    float4 v;
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
-    __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
-    __device__ __forceinline__ float get(int i) const { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-};
-template <> struct Vec<float, 1> {
-    float v;
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(p); }
-    __device__ __forceinline__ void zero() { v = 0.f; }
-    __device__ __forceinline__ float get(int) const { return v; }
-};
-template <> struct Vec<__nv_bfloat16, 8> {
-    uint4 v;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint4*>(p)); }
-    __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
-    __device__ __forceinline__ float get(int i) const
-    {
-        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
-        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));   // bf16 -> fp32 is exact
-    }
-};
-template <> struct Vec<__nv_bfloat16, 1> {
-    unsigned short v;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const unsigned short*>(p)); }
-    __device__ __forceinline__ void zero() { v = 0; }
-    __device__ __forceinline__ float get(int) const { return __uint_as_float((uint32_t)v << 16); }
-};
-
-__device__ __forceinline__ void store_elem(void* out, int out_bf16, int64_t idx, float val)
-{
-    if (out_bf16) static_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(val);
-    else __stcs(static_cast<float*>(out) + idx, val);
-}
 
 #ifndef GNNFD_GATHER_LOADS
 #define GNNFD_GATHER_LOADS 8

@@ -217,7 +217,8 @@ extern "C" int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, 
                                   float negative_slope, float* d_alpha, void* stream)
 {
     using namespace gnnfd;
-    if (!csr || !d_s_src || !d_s_dst || !d_alpha || heads <= 0) return GNNFD_INVALID_ARG;
+    if (!csr || !d_s_src || !d_s_dst || heads <= 0 || (!d_alpha && csr->nnz > 0)) return GNNFD_INVALID_ARG;
+    if (csr->nnz == 0) return GNNFD_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int hh = (heads <= 32 && (heads & (heads - 1)) == 0) ? heads : 1;   // heads handled together
     static const int slots_in_parallel[3] = {2, 8, 32};                       // per degree bin of the row

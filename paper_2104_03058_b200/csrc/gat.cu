@@ -5,10 +5,10 @@
 // the undecomposed one.  The fused kernel walks a row once, keeping a running maximum m, a running
 // denominator l and the un-normalised weighted sum per lane; edge-parallel groups and hub segments
 // are merged by the usual log-sum-exp rule in a fixed order.
-#include <cuda_bf16.h>
 #include <math_constants.h>
 
 #include "schedule.cuh"
+#include "vec.cuh"
 
 namespace gnnfd {
 
@@ -31,36 +31,6 @@ struct GatArgs {
     Range range[kMaxRanges];
 };
 
-template <typename T, int VECN> struct ZVec;
-template <> struct ZVec<float, 4> {
-    float4 v;
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
-    __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
-    __device__ __forceinline__ float get(int i) const { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-};
-template <> struct ZVec<float, 1> {
-    float v;
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(p); }
-    __device__ __forceinline__ void zero() { v = 0.f; }
-    __device__ __forceinline__ float get(int) const { return v; }
-};
-template <> struct ZVec<__nv_bfloat16, 8> {
-    uint4 v;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint4*>(p)); }
-    __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
-    __device__ __forceinline__ float get(int i) const
-    {
-        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
-        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
-    }
-};
-template <> struct ZVec<__nv_bfloat16, 1> {
-    unsigned short v;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const unsigned short*>(p)); }
-    __device__ __forceinline__ void zero() { v = 0; }
-    __device__ __forceinline__ float get(int) const { return __uint_as_float((uint32_t)v << 16); }
-};
-
 __device__ __forceinline__ float widen(float x) { return x; }
 __device__ __forceinline__ float widen(__nv_bfloat16 x) { return __bfloat162float(x); }
 
@@ -70,12 +40,6 @@ __device__ __forceinline__ float leaky(float x, float slope) { return x >= 0.f ?
 __device__ __forceinline__ float merge_scale(float m, float m_new)
 {
     return m == -CUDART_INF_F ? 0.f : expf(m - m_new);
-}
-
-__device__ __forceinline__ void store_out(void* out, int out_bf16, int64_t idx, float val)
-{
-    if (out_bf16) static_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(val);
-    else __stcs(static_cast<float*>(out) + idx, val);
 }
 
 // ------------------------------------------------------------------ scores
@@ -186,7 +150,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         __syncwarp();
 #pragma unroll
         for (int s0 = 0; s0 < SPB; s0 += UB) {
-            ZVec<T, VECN> v[UB][VPL];
+            Vec<T, VECN> v[UB][VPL];
             float lg[UB];
             bool valid[UB];
 #pragma unroll
@@ -272,7 +236,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
             const int64_t o = (int64_t)row * a.ldo + j;
 #pragma unroll
             for (int i = 0; i < VECN; ++i)
-                if (j + i < chunk_end) store_out(a.out, a.out_bf16, o + i, acc[q][i] * inv);
+                if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[q][i] * inv);
         }
     }
 }
@@ -348,7 +312,7 @@ gat_hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict_
     den = 0.f;
 #pragma unroll
     for (int w = 0; w < kReduceWays; ++w) { num += s_num[w][c]; den += s_den[w][c]; }
-    store_out(out, out_bf16, (int64_t)row * ldo + j, den > 0.f ? num / den : 0.f);
+    store_elem(out, out_bf16, (int64_t)row * ldo + j, den > 0.f ? num / den : 0.f);
 }
 
 // ------------------------------------------------------------------ host side

@@ -365,3 +365,66 @@ def test_chunk_width_tuner_picks_a_candidate_and_leaves_a_valid_result(g):
     assert width_sage in (64, 602)
     with pytest.raises(g.GnnfdError):
         g.tune_chunk_width(csr, xd, "gcn", f=w.f, candidates=[0])
+
+
+# ------------------------------------------------------------------ degenerate shapes
+
+def test_degenerate_shapes(g):
+    # a single vertex with a self-loop, one feature column
+    one = np.zeros(1, np.int32)
+    csr = g.build_csr(1, dev(one), dev(one), 0)
+    x = torch.tensor([[2.5]], device="cuda")
+    assert g.aggregate_gcn(csr, x, f=1, chunk_width=1).item() == 2.5
+    assert g.aggregate_sage(csr, x, f=1, chunk_width=7).item() == 2.5
+    # no edges at all: every row is empty and the output is zero, not stale memory
+    empty = np.zeros(0, np.int32)
+    csr = g.build_csr(9, dev(empty), dev(empty), 0)
+    out = torch.full((9, 5), 3.0, device="cuda")
+    g.aggregate_gcn(csr, torch.ones((9, 5), device="cuda"), f=5, chunk_width=2, out=out)
+    assert bool((out == 0).all())
+    a = torch.ones((1, 5), device="cuda")
+    out.fill_(3.0)
+    g.aggregate_gat(csr, torch.ones((9, 5), device="cuda"), a, a, 1, 5, 0.2, chunk_width=5, out=out)
+    assert bool((out == 0).all())
+    assert g.edge_softmax(csr, torch.zeros((9, 2), device="cuda"), torch.zeros((9, 2), device="cuda")).shape == (0, 2)
+
+
+@pytest.mark.parametrize("width", [1, 2, 5])
+def test_chunk_width_one_and_odd_widths(g, width):
+    n, f = 2000, 5
+    src, dst = gg.powerlaw_graph(n, 20_000, 2.1, None, 11)
+    x = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=11)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, SL)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    for model, fn in (("gcn", g.aggregate_gcn), ("sage", g.aggregate_sage)):
+        want, scale = orc.aggregate(model, row_ptr, col, x, f)
+        assert_close_f32(fn(csr, dev(x), f=f, chunk_width=width).cpu().numpy(), want, scale, "%s width %d" % (model, width))
+
+
+@pytest.mark.parametrize("heads,dim", [(40, 2), (6, 1), (33, 4)])
+def test_gat_many_and_odd_head_counts(g, heads, dim):
+    n = 3000
+    src, dst = gg.powerlaw_graph(n, 40_000, 2.1, None, heads)
+    dst[:2500] = 9                      # a hub row
+    f = heads * dim
+    z = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=heads)
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=heads, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=heads, stream=6)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, SL)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    want, scale = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2, threads=orc.max_threads())
+    for width in (f, 8):
+        got = g.aggregate_gat(csr, dev(z), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
+        assert_close_f32(got.cpu().numpy(), want, scale, "gat %dx%d width %d" % (heads, dim, width))
+    s_src, s_dst = g.gat_scores(dev(z), dev(a_src), dev(a_dst), heads, dim)
+    alpha = g.edge_softmax(csr, s_src, s_dst, 0.2).cpu().numpy()
+    want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), 0.2)
+    assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
+
+
+def test_int64_ids_beyond_int32_are_rejected(g):
+    src = torch.tensor([0, 2 ** 31 + 5], dtype=torch.int64, device="cuda")
+    dst = torch.tensor([1, 2], dtype=torch.int64, device="cuda")
+    with pytest.raises(g.GnnfdError) as err:
+        g.build_csr(10, src, dst, 0)
+    assert err.value.status == g.BAD_INDEX
