@@ -51,6 +51,13 @@ WORKLOADS = {
     "config5_f16": (lambda s: gg.config5(s, f=16), 16, "GCN, RMAT scale 21 (as config5_f256), F=16 bf16"),
     "config5_f8": (lambda s: gg.config5(s, f=8), 8, "GCN, RMAT scale 21 (as config5_f256), F=8 bf16"),
 }
+# hidden-layer aggregation on the config-4 graph (the paper's Hid = 8 / 16 / 32 / 64 settings, Section III)
+for _model in ("gcn", "sage", "gat"):
+    for _hid in (8, 16, 32, 64):
+        WORKLOADS["reddit_%s_hid%d" % (_model, _hid)] = (
+            (lambda s, m=_model, h=_hid: gg.reddit_hidden(m, h, s)), _hid,
+            "%s on the config-4 graph (232,965 vertices, ~115M edges + self-loops), hidden width %d fp32"
+            % (_model.upper(), _hid))
 # DRAM bytes per launch of the dominant kernel from a one-pass ncu capture of the same launch
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources they were taken with.
 NCU_TRAFFIC = {"config4": {"bytes": 16.83e9, "sources_sha1": "04e27ab764e4f89b402d58e5b892ff68df2474d4"}}

@@ -226,3 +226,21 @@ def scaled(config: str, factor: float, seed: int = 0) -> Workload:
         scale = max(8, 21 + int(round(np.log2(factor))))
         return config5(seed, scale=scale, edges=max(1024, int(60_000_000 * factor)), f=f)
     raise ValueError(config)
+
+
+def reddit_hidden(model: str = "gcn", hidden: int = 32, seed: int = 0, dim: int = 8) -> Workload:
+    """Hidden-layer aggregation on the Reddit-shaped graph of config 4 (the paper's Hid = 8 / 16 / 32 / 64
+    settings of Section III): same graph and self-loops, features [n, hidden] fp32 N(0,1).  For GAT the
+    hidden width is split into heads of ``dim`` columns (one head when hidden <= dim)."""
+    n = 232_965
+    src, dst = powerlaw_graph(n, 114_615_892, 2.1, 20_000, seed)
+    x = features_f32(n, hidden, dist="normal", p0=0.0, p1=1.0, seed=seed)
+    if model == "gat":
+        d = min(dim, hidden)
+        heads = hidden // d
+        a_src = features_f32(heads, d, dist="normal", p0=0.0, p1=0.1, seed=seed, stream=5)
+        a_dst = features_f32(heads, d, dist="normal", p0=0.0, p1=0.1, seed=seed, stream=6)
+        return Workload("reddit_gat_hid%d" % hidden, "gat", n, src, dst, FLAG_SELF_LOOPS, hidden, hidden, x, "f32",
+                        tuple(sorted({d, hidden})), heads=heads, dim=d, a_src=a_src, a_dst=a_dst, negative_slope=0.2)
+    return Workload("reddit_%s_hid%d" % (model, hidden), model, n, src, dst, FLAG_SELF_LOOPS, hidden, hidden, x, "f32",
+                    tuple(sorted({min(hidden, 8), hidden})))

@@ -70,3 +70,27 @@ def test_config4_tuner_prefers_a_decomposed_sweep(big):
     width, ms = g.tune_chunk_width(csr, xd, "gcn", f=w.f, candidates=[602, 128, 64, 32], out=out[:, :w.f])
     # the slice gathered per sweep must fit L2: the undecomposed sweep (561 MB) and very narrow chunks lose
     assert width in (64, 128) and 5.0 < ms < 60.0
+
+
+def test_config4_graph_gat_and_sage_hidden64_sampled_rows(big):
+    """The paper's GAT / GraphSAGE setting on the Reddit-shaped graph (hidden width 64): sampled rows,
+    the hub rows among them, against the oracle; chunk width 8 is the paper's GAT granularity."""
+    g, w, csr, (row_ptr, col, _) = big
+    deg = np.diff(row_ptr)
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([rng.choice(w.n, 96, replace=False), np.argsort(deg)[-8:]])).astype(np.int64)
+    heads, dim = 8, 8
+    z = gg.features_f32(w.n, heads * dim, dist="normal", p0=0.0, p1=1.0, seed=1)
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0.0, p1=0.1, seed=1, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0.0, p1=0.1, seed=1, stream=6)
+    zd = torch.from_numpy(z).cuda()
+    sel = torch.from_numpy(rows).cuda()
+    want, scale = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2, rows=rows, threads=orc.max_threads())
+    for width in (8, 64):
+        got = g.aggregate_gat(csr, zd, torch.from_numpy(a_src).cuda(), torch.from_numpy(a_dst).cuda(), heads, dim, 0.2,
+                              chunk_width=width)[sel].cpu().numpy()
+        assert (np.abs(got - want) <= 1e-5 * scale + 1e-6).all(), "gat width %d" % width
+    want, scale = orc.aggregate("sage", row_ptr, col, z, heads * dim, rows=rows, threads=orc.max_threads())
+    for width in (4, 64):
+        got = g.aggregate_sage(csr, zd, f=heads * dim, chunk_width=width)[sel].cpu().numpy()
+        assert (np.abs(got - want) <= 1e-5 * scale + 1e-6).all(), "sage width %d" % width
