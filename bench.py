@@ -235,6 +235,8 @@ def run_ours(args):
     device = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
+    if not os.path.exists(g.build.LIB_PATH):      # a checkout without the built library: compile it (atomic replace)
+        g.build.build_library()
     g.lib()
 
     w = make_workload(args.workload, args.seed + rank)
