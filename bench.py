@@ -107,7 +107,7 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as fh:
             return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+    return 6650.0, "fallback (6.65 TB/s, an earlier copy-bandwidth measurement on the same GPU model)"
 
 
 class ClockSampler:
