@@ -83,10 +83,23 @@ radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int mask, in
     h[threadIdx.x + kThreads] = 0;
     __syncthreads();
     const int64_t base = (int64_t)blockIdx.x * kSortTile;
+    if (base + kSortTile <= m) {
+        // full tile: 16-byte loads, all of them issued before the first shared-memory atomic
+        const ulonglong2* k2 = reinterpret_cast<const ulonglong2*>(keys + base);
+        ulonglong2 v[kSortItems / 2];
 #pragma unroll
-    for (int i = 0; i < kSortItems; ++i) {
-        const int64_t idx = base + i * kThreads + threadIdx.x;
-        if (idx < m) atomicAdd(&h[(int)(keys[idx] >> shift) & mask], 1);
+        for (int i = 0; i < kSortItems / 2; ++i) v[i] = __ldcs(k2 + i * kThreads + threadIdx.x);
+#pragma unroll
+        for (int i = 0; i < kSortItems / 2; ++i) {
+            atomicAdd(&h[(int)(v[i].x >> shift) & mask], 1);
+            atomicAdd(&h[(int)(v[i].y >> shift) & mask], 1);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < kSortItems; ++i) {
+            const int64_t idx = base + i * kThreads + threadIdx.x;
+            if (idx < m) atomicAdd(&h[(int)(keys[idx] >> shift) & mask], 1);
+        }
     }
     __syncthreads();
     hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
