@@ -428,3 +428,26 @@ def test_int64_ids_beyond_int32_are_rejected(g):
     with pytest.raises(g.GnnfdError) as err:
         g.build_csr(10, src, dst, 0)
     assert err.value.status == g.BAD_INDEX
+
+
+# ------------------------------------------------------------------ sort boundaries
+
+@pytest.mark.parametrize("n,e,flags", [
+    (4096, 4096, 0), (4097, 8191, DD), (255, 4095, SL | DD), (256, 4097, SY), (257, 12288, SY | DD | SL),
+    (1, 5000, DD), (2, 4096 * 3 + 1, 0), (513, 511, SL),
+    ((1 << 20) + 1, 3000, DD),            # 21 + 21 key bits, values packed beside them
+    (1 << 22, 4000, SY),                  # 22 + 23 key bits, still one word
+    (1 << 27, 2000, DD),                  # 27 + 28 key bits: keys and values travel separately
+])
+def test_csr_sort_boundaries(g, n, e, flags):
+    src, dst = gg.uniform_graph(n, e, seed=n % 1000 + e)
+    if n > 4:
+        dst[: e // 3] = dst[0]            # a long run of equal destinations, with duplicates of (dst, src)
+        src[: e // 6] = src[0]
+    csr = g.build_csr(n, dev(src), dev(dst), flags)
+    row_ptr, col, perm = orc.build_csr(n, src, dst, flags)
+    assert csr.nnz == len(col)
+    assert torch.equal(csr.row_ptr.cpu(), torch.from_numpy(row_ptr))
+    assert torch.equal(csr.col_idx.cpu(), torch.from_numpy(col))
+    assert torch.equal(csr.perm.cpu(), torch.from_numpy(perm))
+    assert sum(csr.bin_count) == n
