@@ -201,9 +201,16 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
                         float negative_slope, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
                         int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
 
-/* alpha[k, h] for every CSR slot k, [nnz, heads] fp32 in CSR order, from caller-supplied scores. */
+/* Materialised edge softmax: alpha[k, h] for every CSR slot k, [nnz, heads] fp32 in CSR order, from
+ * caller-supplied scores d_s_src / d_s_dst [n, heads] fp32 (logit and softmax as defined above).
+ * d_scratch: per-call buffer of gnnfd_edge_softmax_workspace_bytes(csr, heads) bytes (the running
+ * maximum and sum of every hub-row segment; 0 bytes when the graph has no hub row, NULL is then
+ * accepted), 8-byte aligned.  16-byte-aligned pointers with heads a multiple of 4 take the 128-bit
+ * path; anything else is still correct through narrower accesses.  The call only enqueues work. */
+int gnnfd_edge_softmax_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, size_t* scratch_bytes);
+
 int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
-                       float negative_slope, float* d_alpha, void* stream);
+                       float negative_slope, float* d_alpha, void* d_scratch, size_t scratch_bytes, void* stream);
 
 /* ------------------------------------------------------------------ diagnostics */
 

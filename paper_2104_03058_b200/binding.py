@@ -61,7 +61,8 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_gat_scores.argtypes = [i64, vp, i64, i32, vp, vp, i32, i32, vp, vp, vp]
         L.gnnfd_gat_workspace_bytes.argtypes = [vp, i32, i32, pp(sz)]
         L.gnnfd_aggregate_gat.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32, vp, sz, vp]
-        L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp]
+        L.gnnfd_edge_softmax_workspace_bytes.argtypes = [vp, i32, pp(sz)]
+        L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp, sz, vp]
         L.gnnfd_status_string.argtypes = [ctypes.c_int]
         L.gnnfd_status_string.restype = ctypes.c_char_p
         L.gnnfd_last_cuda_error.restype = ctypes.c_int
@@ -313,8 +314,15 @@ def aggregate_gat(csr: Csr, z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.T
     return out
 
 
+def edge_softmax_workspace_bytes(csr: Csr, heads: int) -> int:
+    s = ctypes.c_size_t()
+    _check(lib().gnnfd_edge_softmax_workspace_bytes(csr.handle, heads, ctypes.byref(s)),
+           "gnnfd_edge_softmax_workspace_bytes")
+    return s.value
+
+
 def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_slope: float = 0.2,
-                 out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+                 out: torch.Tensor | None = None, scratch=None, stream=None) -> torch.Tensor:
     heads = s_src.shape[1]
     s_src = s_src.contiguous()
     s_dst = s_dst.contiguous()
@@ -322,8 +330,12 @@ def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_sl
         raise TypeError("scores must be float32 [n, heads]")
     if out is None:
         out = torch.empty((csr.nnz, heads), dtype=torch.float32, device=s_src.device)
+    if scratch is None:
+        scratch = _alloc_bytes(edge_softmax_workspace_bytes(csr, heads), s_src.device)
     _check(lib().gnnfd_edge_softmax(csr.handle, ctypes.c_void_p(s_src.data_ptr()), ctypes.c_void_p(s_dst.data_ptr()),
-                                    heads, negative_slope, ctypes.c_void_p(out.data_ptr()), _stream_ptr(stream)),
+                                    heads, negative_slope, ctypes.c_void_p(out.data_ptr()),
+                                    ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
+                                    _stream_ptr(stream)),
            "gnnfd_edge_softmax")
     return out
 

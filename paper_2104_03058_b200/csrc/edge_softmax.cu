@@ -1,246 +1,325 @@
 // Materialised edge softmax: alpha[k, h] for every CSR slot k from caller-supplied scores.
 //
 // Logit of slot k of row v, head h: LeakyReLU(s_src[col_idx[k], h] + s_dst[v, h]); alpha is the softmax
-// over the slots of the row.  A row is shared by S threads.  When heads is a power of two <= 32 a
-// thread owns head t % heads and every (S / heads)-th slot, so consecutive threads write
-// consecutive addresses of alpha; otherwise the heads are taken one at a time.  S grows with the
-// degree class of the row (the rows come sorted by degree, so a warp's rows have similar lengths).
-// Rows of the top degree bin get a block each and hub rows a whole thread-block cluster: the per-head
-// maxima and sums of the member blocks are exchanged through distributed shared memory.
-#include <cooperative_groups.h>
+// over the slots of the row.  The work is cut exactly as in the gather kernels: rows come sorted by
+// degree class and a row is shared by S lanes (1 / 4 / 8 / 32 by class); a hub row is cut into segments
+// of GNNFD_HUB_SEGMENT slots, one warp each, so that no unit of work is longer than a segment.  A lane
+// owns whole slots: it loads the HB heads of a slot's source score with one or two 16-byte loads and
+// writes the HB alphas of the slot the same way, so the reads of col_idx and the writes of alpha are
+// contiguous across the lanes of a row.
+//
+// An ordinary row is done by its lanes in one go: a running (max, sum) over the row, a fixed
+// butterfly merge across the lanes, then the write pass (the logits stay in registers when the row
+// fits one batch, otherwise they are gathered again: the row's indices and scores are cache hits).
+// Hub rows take three launches: per-segment (max, sum), a merge per row in ascending segment order,
+// and the write pass per segment.  Nothing waits on another block and nothing is accumulated
+// atomically, so the result is the same bit for bit from run to run.
+//
+// The exponentials are base-2 (logits pre-multiplied by log2 e): the argument is rounded once more
+// than with expf, which moves a result by about |logit| * 6e-8 relative (the fp32 sum s_src + s_dst
+// already carries an error of that size).
 #include <math_constants.h>
 
-#include "common.cuh"
-
-namespace cg = cooperative_groups;
+#include "schedule.cuh"
 
 namespace gnnfd {
 
-constexpr int kRowBlock = 256;          // threads per block, ordinary rows
-constexpr int kBigBlock = 256;          // threads per block, rows of 129 .. GNNFD_HUB_DEGREE entries (one block each)
-constexpr int kHubBlock = 1024;         // threads per block, hub rows
-constexpr int kHubCluster = 8;          // blocks per hub row
+constexpr int kSlotsInFlight = 4;                  // slots a lane has in flight
+constexpr float kLog2e = 1.4426950408889634f;
 
-__device__ __forceinline__ float leaky_relu(float x, float slope) { return x >= 0.f ? x : slope * x; }
-
-struct RowView {
+struct SoftmaxArgs {
+    const int32_t* row_ptr;
     const int32_t* col_idx;
+    const int32_t* row_order;
+    const int32_t* seg_row;
+    const int32_t* seg_begin;
+    const int32_t* hub_seg_ptr;
     const float* s_src;
+    const float* s_dst;
     float* alpha;
-    int32_t b, e;
-    int heads;
+    float2* seg_stats;       // [n_segments, heads]: (max, sum) of a segment, later (max, 1 / sum) of its row
     float slope;
+    int32_t heads;
+    int32_t n_hub;
+    int32_t n_ranges;
+    Range range[kMaxRanges];
 };
 
-// logit of slot k, head h
-__device__ __forceinline__ float logit(const RowView& r, int32_t k, int h, float sd)
-{
-    return leaky_relu(__ldg(r.s_src + (int64_t)__ldg(r.col_idx + k) * r.heads + h) + sd, r.slope);
-}
+enum { kModeRows = 0, kModeHubStats = 1, kModeHubWrite = 2 };
 
-// Running maximum and denominator over slots first, first + step, ... (kInFlight logits in flight).
-constexpr int kInFlight = 8;
-__device__ __forceinline__ void online_max_sum(const RowView& r, int32_t first, int step, int h, float sd, float* m_out,
-                                               float* l_out)
+template <int HB>
+__device__ __forceinline__ void load_heads(const float* p, float (&v)[HB])
 {
-    float m = -CUDART_INF_F, l = 0.f;
-    for (int32_t k = first; k < r.e; k += kInFlight * step) {
-        float t[kInFlight];
+    if constexpr (HB % 4 == 0) {
 #pragma unroll
-        for (int i = 0; i < kInFlight; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : -CUDART_INF_F;
-        float mx = m;                                                               // t[0] is valid, so mx ends finite
-#pragma unroll
-        for (int i = 0; i < kInFlight; ++i) mx = fmaxf(mx, t[i]);
-        l *= expf(m - mx);
-#pragma unroll
-        for (int i = 0; i < kInFlight; ++i) l += expf(t[i] - mx);                   // exp(-inf) = 0 for the missing ones
-        m = mx;
-    }
-    *m_out = m;
-    *l_out = l;
-}
-
-__device__ __forceinline__ void write_alpha(const RowView& r, int32_t first, int step, int h, float sd, float m, float inv)
-{
-    for (int32_t k = first; k < r.e; k += kInFlight * step) {
-        float t[kInFlight];
-#pragma unroll
-        for (int i = 0; i < kInFlight; ++i) t[i] = k + i * step < r.e ? logit(r, k + i * step, h, sd) : 0.f;
-#pragma unroll
-        for (int i = 0; i < kInFlight; ++i)
-            if (k + i * step < r.e) __stcs(r.alpha + (int64_t)(k + i * step) * r.heads + h, expf(t[i] - m) * inv);
+        for (int i = 0; i < HB; i += 4) {
+            const float4 q = __ldg(reinterpret_cast<const float4*>(p + i));
+            v[i] = q.x; v[i + 1] = q.y; v[i + 2] = q.z; v[i + 3] = q.w;
+        }
+    } else if constexpr (HB == 2) {
+        const float2 q = __ldg(reinterpret_cast<const float2*>(p));
+        v[0] = q.x; v[1] = q.y;
+    } else {
+        v[0] = __ldg(p);
     }
 }
 
-// ---- ordinary rows: S lanes of a warp per row
-
-template <int S>
-__global__ void __launch_bounds__(kRowBlock)
-edge_softmax_rows(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                  const int32_t* __restrict__ rows, int64_t n_rows, const float* __restrict__ s_src,
-                  const float* __restrict__ s_dst, int heads, int hh, float slope, float* __restrict__ alpha)
+template <int HB>
+__device__ __forceinline__ void store_heads(float* p, const float (&v)[HB])
 {
-    const int64_t slot = (int64_t)blockIdx.x * (kRowBlock / S) + threadIdx.x / S;
-    const int sl = threadIdx.x % S;
-    const bool active = slot < n_rows;
-    const int32_t row = active ? rows[slot] : 0;
-    RowView r{col_idx, s_src, alpha, active ? row_ptr[row] : 0, active ? row_ptr[row + 1] : 0, heads, slope};
-    const int step = S / hh;
-    for (int h0 = 0; h0 < heads; h0 += hh) {
-        const int h = h0 + sl % hh;
-        const float sd = active ? s_dst[(int64_t)row * heads + h] : 0.f;
-        const int32_t first = r.b + sl / hh;
-        if (__all_sync(0xffffffffu, r.e - r.b <= kInFlight * step)) {
-            // every row of this warp fits one round: the logits stay in registers between the two phases
-            float t[kInFlight];
-            float m = -CUDART_INF_F;
+    if constexpr (HB % 4 == 0) {
 #pragma unroll
-            for (int i = 0; i < kInFlight; ++i) {
-                t[i] = first + i * step < r.e ? logit(r, first + i * step, h, sd) : -CUDART_INF_F;
-                m = fmaxf(m, t[i]);
+        for (int i = 0; i < HB; i += 4) __stcs(reinterpret_cast<float4*>(p + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+    } else if constexpr (HB == 2) {
+        __stcs(reinterpret_cast<float2*>(p), make_float2(v[0], v[1]));
+    } else {
+        __stcs(p, v[0]);
+    }
+}
+
+// share of a partial result with maximum m under the merged maximum mx
+__device__ __forceinline__ float rescale(float m, float mx) { return m == -CUDART_INF_F ? 0.f : exp2f(m - mx); }
+
+// base-2 logits of up to kSlotsInFlight slots k, k + S, ... of one row; missing slots get -inf
+template <int HB, int S>
+__device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const float* ssrc, const float (&sd)[HB], int32_t k,
+                                            int32_t e, float (&t)[kSlotsInFlight][HB])
+{
+    int32_t u[kSlotsInFlight];
+#pragma unroll
+    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = k + i * S < e ? __ldg(a.col_idx + k + i * S) : -1;
+#pragma unroll
+    for (int i = 0; i < kSlotsInFlight; ++i) {
+        if (u[i] >= 0) {
+            load_heads<HB>(ssrc + (int64_t)u[i] * a.heads, t[i]);
+        } else {
+#pragma unroll
+            for (int h = 0; h < HB; ++h) t[i][h] = 0.f;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kSlotsInFlight; ++i)
+#pragma unroll
+        for (int h = 0; h < HB; ++h) {
+            const float x = t[i][h] + sd[h];
+            t[i][h] = u[i] >= 0 ? (x >= 0.f ? x : a.slope * x) * kLog2e : -CUDART_INF_F;
+        }
+}
+
+template <int HB, int S, int MODE>
+__device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range& rg, int block_in_range)
+{
+    constexpr unsigned kFull = 0xffffffffu;
+    const int tid = threadIdx.x;
+    const int slot = block_in_range * (kBlock / S) + tid / S;
+    const int sl = tid % S;
+    const bool active = slot < rg.item_count;
+    int32_t row = 0, b = 0, e = 0;
+    if (active) {
+        if (rg.hub) {
+            row = a.seg_row[slot];
+            b = a.seg_begin[slot];
+            e = min(b + kHubSegment, a.row_ptr[row + 1]);
+        } else {
+            row = a.row_order[rg.item_begin + slot];
+            b = a.row_ptr[row];
+            e = a.row_ptr[row + 1];
+        }
+    }
+    // every row of the warp fits one batch: the write pass reuses the logits of the first pass
+    const bool fits = MODE == kModeRows && __all_sync(kFull, e - b <= S * kSlotsInFlight);
+
+    for (int h0 = 0; h0 < a.heads; h0 += HB) {
+        float sd[HB];
+#pragma unroll
+        for (int h = 0; h < HB; ++h) sd[h] = 0.f;
+        if (active) load_heads<HB>(a.s_dst + (int64_t)row * a.heads + h0, sd);
+        const float* ssrc = a.s_src + h0;
+        float m[HB], inv[HB];
+        float t[kSlotsInFlight][HB];
+
+        if (MODE != kModeHubWrite) {
+            float l[HB];
+#pragma unroll
+            for (int h = 0; h < HB; ++h) { m[h] = -CUDART_INF_F; l[h] = 0.f; }
+            for (int32_t k = b + sl; k < e; k += S * kSlotsInFlight) {
+                load_logits<HB, S>(a, ssrc, sd, k, e, t);
+#pragma unroll
+                for (int h = 0; h < HB; ++h) {
+                    float mx = m[h];                                   // t[0] is a real slot, so mx ends finite
+#pragma unroll
+                    for (int i = 0; i < kSlotsInFlight; ++i) mx = fmaxf(mx, t[i][h]);
+                    float sum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < kSlotsInFlight; ++i) sum += exp2f(t[i][h] - mx);      // 2^-inf = 0
+                    l[h] = l[h] * rescale(m[h], mx) + sum;
+                    m[h] = mx;
+                }
+            }
+            // butterfly over the S lanes of the row; both partners evaluate the same commutative expression
+            if constexpr (S > 1) {
+#pragma unroll
+                for (int o = S / 2; o >= 1; o >>= 1)
+#pragma unroll
+                    for (int h = 0; h < HB; ++h) {
+                        const float mo = __shfl_xor_sync(kFull, m[h], o);
+                        const float lo = __shfl_xor_sync(kFull, l[h], o);
+                        const float mx = fmaxf(m[h], mo);
+                        l[h] = __fadd_rn(__fmul_rn(l[h], rescale(m[h], mx)), __fmul_rn(lo, rescale(mo, mx)));
+                        m[h] = mx;
+                    }
+            }
+            if (MODE == kModeHubStats) {
+                if (active && sl == 0) {
+#pragma unroll
+                    for (int h = 0; h < HB; ++h) a.seg_stats[(int64_t)slot * a.heads + h0 + h] = make_float2(m[h], l[h]);
+                }
+                continue;
             }
 #pragma unroll
-            for (int o = S / 2; o >= 1; o >>= 1)
-                if (o >= hh) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            float l = 0.f;
+            for (int h = 0; h < HB; ++h) inv[h] = 1.f / l[h];          // unused (inf) for an empty row
+        } else {
 #pragma unroll
-            for (int i = 0; i < kInFlight; ++i) {
-                t[i] = first + i * step < r.e ? expf(t[i] - m) : 0.f;
-                l += t[i];
+            for (int h = 0; h < HB; ++h) {
+                const float2 st = active ? a.seg_stats[(int64_t)slot * a.heads + h0 + h] : make_float2(0.f, 0.f);
+                m[h] = st.x;
+                inv[h] = st.y;
             }
-#pragma unroll
-            for (int o = S / 2; o >= 1; o >>= 1)
-                if (o >= hh) l += __shfl_xor_sync(0xffffffffu, l, o);
-            const float inv = 1.f / l;
-#pragma unroll
-            for (int i = 0; i < kInFlight; ++i)
-                if (first + i * step < r.e) __stcs(alpha + (int64_t)(first + i * step) * heads + h, t[i] * inv);
-            continue;
         }
-        float m, l;
-        online_max_sum(r, first, step, h, sd, &m, &l);
-        float mall = m;
-#pragma unroll
-        for (int o = S / 2; o >= 1; o >>= 1)
-            if (o >= hh) mall = fmaxf(mall, __shfl_xor_sync(0xffffffffu, mall, o));
-        l = m == -CUDART_INF_F ? 0.f : l * expf(m - mall);
-#pragma unroll
-        for (int o = S / 2; o >= 1; o >>= 1)
-            if (o >= hh) l += __shfl_xor_sync(0xffffffffu, l, o);
-        write_alpha(r, first, step, h, sd, mall, 1.f / l);
-    }
-}
 
-// ---- long rows: one block, hub rows: one cluster of blocks per row
-
-// Combines one value per thread over all threads of the cluster that own the same head (threads with
-// equal t % hh; hh divides 32).  `mine` is this block's exchange buffer of 32 floats.
-template <bool IS_MAX, int THREADS, int CLUSTER>
-__device__ __forceinline__ float cluster_combine(float v, int hh, float* warp_buf, float* mine, cg::cluster_group& cluster)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (fits) {
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1)
-        if (o >= hh) {
-            const float other = __shfl_xor_sync(0xffffffffu, v, o);
-            v = IS_MAX ? fmaxf(v, other) : v + other;
+            for (int i = 0; i < kSlotsInFlight; ++i) {
+                const int32_t k = b + sl + i * S;
+                if (k < e) {
+                    float w[HB];
+#pragma unroll
+                    for (int h = 0; h < HB; ++h) w[h] = exp2f(t[i][h] - m[h]) * inv[h];
+                    store_heads<HB>(a.alpha + (int64_t)k * a.heads + h0, w);
+                }
+            }
+        } else {
+            for (int32_t k = b + sl; k < e; k += S * kSlotsInFlight) {
+                load_logits<HB, S>(a, ssrc, sd, k, e, t);
+#pragma unroll
+                for (int i = 0; i < kSlotsInFlight; ++i) {
+                    if (k + i * S < e) {
+                        float w[HB];
+#pragma unroll
+                        for (int h = 0; h < HB; ++h) w[h] = exp2f(t[i][h] - m[h]) * inv[h];
+                        store_heads<HB>(a.alpha + (int64_t)(k + i * S) * a.heads + h0, w);
+                    }
+                }
+            }
         }
-    __syncthreads();                                  // the previous combine's readers are done
-    warp_buf[warp * 32 + lane] = v;
-    __syncthreads();
-    float acc = warp_buf[lane];
-#pragma unroll
-    for (int w = 1; w < THREADS / 32; ++w) {
-        const float other = warp_buf[w * 32 + lane];
-        acc = IS_MAX ? fmaxf(acc, other) : acc + other;
-    }
-    if (CLUSTER == 1) return acc;
-    if (warp == 0) mine[lane] = acc;
-    cluster.sync();                                   // every block's `mine` is complete
-    acc = IS_MAX ? -CUDART_INF_F : 0.f;
-#pragma unroll
-    for (int rk = 0; rk < CLUSTER; ++rk) {
-        const float other = cluster.map_shared_rank(mine, rk)[lane];
-        acc = IS_MAX ? fmaxf(acc, other) : acc + other;
-    }
-    cluster.sync();                                   // all reads done before the buffers are reused
-    return acc;
-}
-
-template <int THREADS, int CLUSTER>
-__global__ void __cluster_dims__(CLUSTER, 1, 1) __launch_bounds__(THREADS)
-edge_softmax_big(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                 const int32_t* __restrict__ rows, const float* __restrict__ s_src, const float* __restrict__ s_dst,
-                 int heads, int hh, float slope, int32_t min_len, int32_t max_len, float* __restrict__ alpha)
-{
-    __shared__ float warp_buf[THREADS];
-    __shared__ float mine[32];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int32_t row = rows[blockIdx.x / CLUSTER];
-    {   // rows outside [min_len, max_len] belong to another launch; the whole cluster leaves together
-        const int32_t len = row_ptr[row + 1] - row_ptr[row];
-        if (len < min_len || len > max_len) return;
-    }
-    const int t = (CLUSTER == 1 ? 0 : (int)cluster.block_rank() * THREADS) + threadIdx.x;
-    RowView r{col_idx, s_src, alpha, row_ptr[row], row_ptr[row + 1], heads, slope};
-    const int step = THREADS * CLUSTER / hh;
-    for (int h0 = 0; h0 < heads; h0 += hh) {
-        const int h = h0 + t % hh;
-        const float sd = s_dst[(int64_t)row * heads + h];
-        float m, l;
-        online_max_sum(r, r.b + t / hh, step, h, sd, &m, &l);
-        const float mall = cluster_combine<true, THREADS, CLUSTER>(m, hh, warp_buf, mine, cluster);
-        l = m == -CUDART_INF_F ? 0.f : l * expf(m - mall);
-        l = cluster_combine<false, THREADS, CLUSTER>(l, hh, warp_buf, mine, cluster);
-        write_alpha(r, r.b + t / hh, step, h, sd, mall, 1.f / l);
     }
 }
 
-typedef void (*RowKernel)(const int32_t*, const int32_t*, const int32_t*, int64_t, const float*, const float*, int, int,
-                          float, float*);
-
-static RowKernel pick_rows(int s)
+// All ordinary rows (stats and write in one go) and, in the same grid, the write pass of the hub segments.
+template <int HB>
+__global__ void __launch_bounds__(kBlock) edge_softmax_rows(const __grid_constant__ SoftmaxArgs a)
 {
-    switch (s) {
-        case 1: return edge_softmax_rows<1>;
-        case 2: return edge_softmax_rows<2>;
-        case 4: return edge_softmax_rows<4>;
-        case 8: return edge_softmax_rows<8>;
-        case 16: return edge_softmax_rows<16>;
-        default: return edge_softmax_rows<32>;
+    const int rb = blockIdx.x;
+    int r = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxRanges; ++i)
+        if (i < a.n_ranges && rb >= a.range[i].first_block) r = i;
+    const Range rg = a.range[r];
+    const int bir = rb - rg.first_block;
+    if (rg.hub) { softmax_items<HB, 32, kModeHubWrite>(a, rg, bir); return; }
+    switch (rg.ep_log2) {
+        case 0: softmax_items<HB, 1, kModeRows>(a, rg, bir); break;
+        case 1: softmax_items<HB, 2, kModeRows>(a, rg, bir); break;
+        case 2: softmax_items<HB, 4, kModeRows>(a, rg, bir); break;
+        case 3: softmax_items<HB, 8, kModeRows>(a, rg, bir); break;
+        case 4: softmax_items<HB, 16, kModeRows>(a, rg, bir); break;
+        default: softmax_items<HB, 32, kModeRows>(a, rg, bir); break;
     }
+}
+
+// (max, sum) of every hub segment; range 0 of the plan is the hub range
+template <int HB>
+__global__ void __launch_bounds__(kBlock) edge_softmax_hub_stats(const __grid_constant__ SoftmaxArgs a)
+{
+    softmax_items<HB, 32, kModeHubStats>(a, a.range[0], blockIdx.x);
+}
+
+// One thread per (hub row, head): merges the segment results in ascending segment order and leaves the
+// row's (max, 1 / sum) in every segment's entry.
+__global__ void __launch_bounds__(kBlock) edge_softmax_hub_merge(const __grid_constant__ SoftmaxArgs a)
+{
+    const int64_t idx = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (idx >= (int64_t)a.n_hub * a.heads) return;
+    const int i = (int)(idx / a.heads), h = (int)(idx % a.heads);
+    const int32_t s0 = a.hub_seg_ptr[i], s1 = a.hub_seg_ptr[i + 1];
+    float m = -CUDART_INF_F;
+    for (int32_t s = s0; s < s1; ++s) m = fmaxf(m, a.seg_stats[(int64_t)s * a.heads + h].x);
+    float l = 0.f;
+    for (int32_t s = s0; s < s1; ++s) {
+        const float2 st = a.seg_stats[(int64_t)s * a.heads + h];
+        l += st.y * rescale(st.x, m);
+    }
+    const float2 row_stats = make_float2(m, 1.f / l);
+    for (int32_t s = s0; s < s1; ++s) a.seg_stats[(int64_t)s * a.heads + h] = row_stats;
+}
+
+static size_t softmax_scratch_bytes(const gnnfd_csr_t* csr, int32_t heads)
+{
+    return align_up((size_t)csr->n_segments * (size_t)heads * sizeof(float2), 256);
+}
+
+template <int HB>
+static int launch_softmax(const gnnfd_csr_t* csr, SoftmaxArgs& a, int64_t blocks, cudaStream_t s)
+{
+    if (csr->n_segments > 0) {
+        const unsigned hub_blocks = (unsigned)((csr->n_segments + kBlock / 32 - 1) / (kBlock / 32));
+        GNNFD_LAUNCH("edge_softmax_hub_stats", s, edge_softmax_hub_stats<HB>, hub_blocks, kBlock, 0, a);
+        const int64_t pairs = (int64_t)a.n_hub * a.heads;
+        GNNFD_LAUNCH("edge_softmax_hub_merge", s, edge_softmax_hub_merge, (unsigned)((pairs + kBlock - 1) / kBlock), kBlock,
+                     0, a);
+    }
+    GNNFD_LAUNCH("edge_softmax_rows", s, edge_softmax_rows<HB>, (unsigned)blocks, kBlock, 0, a);
+    GNNFD_CUDA_CHECK(cudaGetLastError());
+    return GNNFD_OK;
 }
 
 }  // namespace gnnfd
 
-extern "C" int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
-                                  float negative_slope, float* d_alpha, void* stream)
+extern "C" {
+
+int gnnfd_edge_softmax_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, size_t* scratch_bytes)
+{
+    if (!csr || heads <= 0 || !scratch_bytes) return GNNFD_INVALID_ARG;
+    *scratch_bytes = gnnfd::softmax_scratch_bytes(csr, heads);
+    return GNNFD_OK;
+}
+
+int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
+                       float negative_slope, float* d_alpha, void* d_scratch, size_t scratch_bytes, void* stream)
 {
     using namespace gnnfd;
     if (!csr || !d_s_src || !d_s_dst || heads <= 0 || (!d_alpha && csr->nnz > 0)) return GNNFD_INVALID_ARG;
     if (csr->nnz == 0) return GNNFD_OK;
+    const size_t need = softmax_scratch_bytes(csr, heads);
+    if (need > 0 && (!d_scratch || scratch_bytes < need)) return GNNFD_WORKSPACE_TOO_SMALL;
+    if (need > 0 && ((uintptr_t)d_scratch & 7u)) return GNNFD_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int hh = (heads <= 32 && (heads & (heads - 1)) == 0) ? heads : 1;   // heads handled together
-    static const int slots_in_parallel[3] = {2, 8, 32};                       // per degree bin of the row
-    for (int bin = 0; bin < 3; ++bin) {
-        const int64_t rows = csr->bin_count[bin];
-        if (rows == 0) continue;
-        int lanes = hh * slots_in_parallel[bin];
-        if (lanes > 32) lanes = 32;
-        const int rows_per_block = kRowBlock / lanes;
-        const unsigned grid = (unsigned)((rows + rows_per_block - 1) / rows_per_block);
-        GNNFD_LAUNCH("edge_softmax_rows", s, pick_rows(lanes), grid, kRowBlock, 0, csr->row_ptr, csr->col_idx,
-                     csr->row_order + csr->bin_start[bin], rows, d_s_src, d_s_dst, heads, hh, negative_slope, d_alpha);
-    }
-    if (csr->bin_count[3] > 0)
-        GNNFD_LAUNCH("edge_softmax_long_rows", s, (edge_softmax_big<kBigBlock, 1>), (unsigned)csr->bin_count[3], kBigBlock, 0,
-                     csr->row_ptr, csr->col_idx, csr->row_order + csr->bin_start[3], d_s_src, d_s_dst, heads, hh,
-                     negative_slope, 0, 0x7fffffff, d_alpha);
-    const int64_t n_hub = csr->bin_count[4];
-    if (n_hub > 0)
-        GNNFD_LAUNCH("edge_softmax_hubs", s, (edge_softmax_big<kHubBlock, kHubCluster>), (unsigned)(n_hub * kHubCluster),
-                     kHubBlock, 0, csr->row_ptr, csr->col_idx, csr->row_order + csr->bin_start[4], d_s_src, d_s_dst, heads,
-                     hh, negative_slope, 0, 0x7fffffff, d_alpha);
-    GNNFD_CUDA_CHECK(cudaGetLastError());
-    return GNNFD_OK;
+
+    SoftmaxArgs a;
+    a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.row_order = csr->row_order;
+    a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin; a.hub_seg_ptr = csr->hub_seg_ptr;
+    a.s_src = d_s_src; a.s_dst = d_s_dst; a.alpha = d_alpha; a.seg_stats = static_cast<float2*>(d_scratch);
+    a.slope = negative_slope; a.heads = heads; a.n_hub = (int32_t)csr->bin_count[4];
+    const int64_t blocks = plan_ranges(csr, 1, a.range, &a.n_ranges);
+    if (blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
+    if (blocks == 0) return GNNFD_OK;
+
+    // heads a lane handles per load: the widest of 8 / 4 / 2 / 1 that divides heads and keeps every access aligned
+    const uintptr_t ptrs = (uintptr_t)d_s_src | (uintptr_t)d_s_dst | (uintptr_t)d_alpha;
+    if (heads % 8 == 0 && ptrs % 16 == 0) return launch_softmax<8>(csr, a, blocks, s);
+    if (heads % 4 == 0 && ptrs % 16 == 0) return launch_softmax<4>(csr, a, blocks, s);
+    if (heads % 2 == 0 && ptrs % 8 == 0) return launch_softmax<2>(csr, a, blocks, s);
+    return launch_softmax<1>(csr, a, blocks, s);
 }
+
+}  // extern "C"

@@ -94,3 +94,28 @@ def test_config4_graph_gat_and_sage_hidden64_sampled_rows(big):
     for width in (4, 64):
         got = g.aggregate_sage(csr, zd, f=heads * dim, chunk_width=width)[sel].cpu().numpy()
         assert (np.abs(got - want) <= 1e-5 * scale + 1e-6).all(), "sage width %d" % width
+
+
+def test_config4_graph_edge_softmax_sampled_rows(big):
+    """alpha of every slot of sampled rows of the Reddit-shaped graph (8 heads), hub rows and the
+    shortest rows among them, against the oracle run on the sub-CSR of those rows; every row's alphas
+    sum to one."""
+    g, w, csr, (row_ptr, col, _) = big
+    deg = np.diff(row_ptr)
+    rng = np.random.default_rng(6)
+    rows = np.unique(np.concatenate([rng.choice(w.n, 256, replace=False), np.argsort(deg)[-8:],
+                                     np.argsort(deg)[:8]])).astype(np.int64)
+    heads = 8
+    s_src = gg.features_f32(w.n, heads, dist="normal", p0=0.0, p1=1.5, seed=2, stream=5)
+    s_dst = gg.features_f32(w.n, heads, dist="normal", p0=0.0, p1=1.5, seed=2, stream=6)
+    alpha = g.edge_softmax(csr, torch.from_numpy(s_src).cuda(), torch.from_numpy(s_dst).cuda(), 0.2)
+    slots = np.concatenate([np.arange(row_ptr[v], row_ptr[v + 1]) for v in rows])
+    sub_ptr = np.concatenate([[0], np.cumsum(deg[rows])]).astype(np.int32)
+    want = orc.edge_softmax(sub_ptr, col[slots], s_src.astype(np.float64), s_dst[rows].astype(np.float64), 0.2)
+    got = alpha[torch.from_numpy(slots).cuda()].cpu().numpy()
+    assert (np.abs(got - want) <= 1e-5 * want + 1e-7).all()
+    # row sums over the whole graph: segmented sum of alpha by row on the device, in fp64
+    sums = torch.zeros((w.n, heads), dtype=torch.float64, device="cuda")
+    row_of_slot = torch.repeat_interleave(torch.arange(w.n, device="cuda"), torch.from_numpy(deg).cuda().long())
+    sums.index_add_(0, row_of_slot, alpha.double())
+    assert float((sums - 1.0).abs().max()) <= 1e-5
