@@ -58,6 +58,9 @@ for _model in ("gcn", "sage", "gat"):
             (lambda s, m=_model, h=_hid: gg.reddit_hidden(m, h, s)), _hid,
             "%s on the config-4 graph (232,965 vertices, ~115M edges + self-loops), hidden width %d fp32"
             % (_model.upper(), _hid))
+WORKLOADS["reddit_small_gat_hid64"] = (
+    (lambda s: gg.reddit_hidden("gat", 64, s, factor=0.25)), 64,
+    "GAT on the config-4 recipe at 1/4 of the vertices and 1/16 of the edges, 8 heads x 8 dims fp32")
 # DRAM bytes per launch of the dominant kernel from a one-pass ncu capture of the same launch
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources they were taken with.
 NCU_TRAFFIC = {"config4": {"bytes": 16.83e9, "sources_sha1": "04e27ab764e4f89b402d58e5b892ff68df2474d4"}}

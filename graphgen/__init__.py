@@ -228,12 +228,13 @@ def scaled(config: str, factor: float, seed: int = 0) -> Workload:
     raise ValueError(config)
 
 
-def reddit_hidden(model: str = "gcn", hidden: int = 32, seed: int = 0, dim: int = 8) -> Workload:
+def reddit_hidden(model: str = "gcn", hidden: int = 32, seed: int = 0, dim: int = 8, factor: float = 1.0) -> Workload:
     """Hidden-layer aggregation on the Reddit-shaped graph of config 4 (the paper's Hid = 8 / 16 / 32 / 64
     settings of Section III): same graph and self-loops, features [n, hidden] fp32 N(0,1).  For GAT the
-    hidden width is split into heads of ``dim`` columns (one head when hidden <= dim)."""
-    n = 232_965
-    src, dst = powerlaw_graph(n, 114_615_892, 2.1, 20_000, seed)
+    hidden width is split into heads of ``dim`` columns (one head when hidden <= dim).  ``factor`` < 1
+    scales the vertex count by factor and the edge count by factor squared, as ``scaled`` does."""
+    n = max(256, int(232_965 * factor))
+    src, dst = powerlaw_graph(n, max(n, int(114_615_892 * factor * factor)), 2.1, min(20_000, n - 1), seed)
     x = features_f32(n, hidden, dist="normal", p0=0.0, p1=1.0, seed=seed)
     if model == "gat":
         d = min(dim, hidden)

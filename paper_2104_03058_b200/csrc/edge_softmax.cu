@@ -2,11 +2,11 @@
 //
 // Logit of slot k of row v, head h: LeakyReLU(s_src[col_idx[k], h] + s_dst[v, h]); alpha is the softmax
 // over the slots of the row.  The work is cut exactly as in the gather kernels: rows come sorted by
-// degree class and a row is shared by S lanes (1 / 4 / 8 / 32 by class); a hub row is cut into segments
-// of GNNFD_HUB_SEGMENT slots, one warp each, so that no unit of work is longer than a segment.  A lane
-// owns whole slots: it loads the HB heads of a slot's source score with one or two 16-byte loads and
-// writes the HB alphas of the slot the same way, so the reads of col_idx and the writes of alpha are
-// contiguous across the lanes of a row.
+// degree class and a row is shared by more lanes the longer its class; a hub row is cut into segments
+// of GNNFD_HUB_SEGMENT slots, one warp each, so that no unit of work is longer than a segment.  The
+// heads of a slot are spread over LPS adjacent lanes, four heads (one 16-byte access) each, and SP
+// slots are worked on side by side, so the lanes of a row read the scores of a slot and write its
+// alphas as one contiguous piece, and consecutive slots follow each other in memory.
 //
 // An ordinary row is done by its lanes in one go: a running (max, sum) over the row, a fixed
 // butterfly merge across the lanes, then the write pass (the logits stay in registers when the row
@@ -24,7 +24,13 @@
 
 namespace gnnfd {
 
-constexpr int kSlotsInFlight = 4;                  // slots a lane has in flight
+#ifndef GNNFD_SOFTMAX_IN_FLIGHT
+#define GNNFD_SOFTMAX_IN_FLIGHT 4
+#endif
+#ifndef GNNFD_SOFTMAX_MIN_BLOCKS
+#define GNNFD_SOFTMAX_MIN_BLOCKS 4
+#endif
+constexpr int kSlotsInFlight = GNNFD_SOFTMAX_IN_FLIGHT;      // slots a lane has in flight
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct SoftmaxArgs {
@@ -77,20 +83,42 @@ __device__ __forceinline__ void store_heads(float* p, const float (&v)[HB])
     }
 }
 
-// share of a partial result with maximum m under the merged maximum mx
-__device__ __forceinline__ float rescale(float m, float mx) { return m == -CUDART_INF_F ? 0.f : exp2f(m - mx); }
-
-// base-2 logits of up to kSlotsInFlight slots k, k + S, ... of one row; missing slots get -inf
-template <int HB, int S>
-__device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const float* ssrc, const float (&sd)[HB], int32_t k,
-                                            int32_t e, float (&t)[kSlotsInFlight][HB])
+// 2^x by the hardware approximation (2 ulp; results below 2^-126 become 0, 2^-inf = 0)
+__device__ __forceinline__ float ex2(float x)
 {
-    int32_t u[kSlotsInFlight];
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// share of a partial result with maximum m under the merged maximum mx (both may be -inf)
+__device__ __forceinline__ float rescale(float m, float mx) { return m == -CUDART_INF_F ? 0.f : ex2(m - mx); }
+
+// LeakyReLU(x) * log2 e written as c1 * x + c2 * |x| with c1 = log2 e * (1 + slope) / 2 and
+// c2 = log2 e * (1 - slope) / 2: two instructions per logit and no branch, for any slope.
+struct Leaky {
+    float c1, c2;
+    __device__ __forceinline__ explicit Leaky(float slope) : c1(0.5f * kLog2e * (1.f + slope)), c2(0.5f * kLog2e * (1.f - slope)) {}
+    __device__ __forceinline__ float operator()(float x) const { return fmaf(fabsf(x), c2, x * c1); }
+};
+
+// column indices of slots k, k + SP, ... of one row (-1 past the end of the row)
+template <int SP>
+__device__ __forceinline__ void load_cols(const SoftmaxArgs& a, int32_t k, int32_t e, int32_t (&u)[kSlotsInFlight])
+{
 #pragma unroll
-    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = k + i * S < e ? __ldg(a.col_idx + k + i * S) : -1;
+    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = k + i * SP < e ? __ldg(a.col_idx + k + i * SP) : -1;
+}
+
+// base-2 logits of the slots whose column indices are u[].  FULL: all of them exist; otherwise the
+// missing ones (u < 0) get -inf.
+template <int HB, bool FULL>
+__device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const Leaky& leaky, const float* ssrc, const float (&sd)[HB],
+                                            const int32_t (&u)[kSlotsInFlight], float (&t)[kSlotsInFlight][HB])
+{
 #pragma unroll
     for (int i = 0; i < kSlotsInFlight; ++i) {
-        if (u[i] >= 0) {
+        if (FULL || u[i] >= 0) {
             load_heads<HB>(ssrc + (int64_t)u[i] * a.heads, t[i]);
         } else {
 #pragma unroll
@@ -101,18 +129,41 @@ __device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const float* s
     for (int i = 0; i < kSlotsInFlight; ++i)
 #pragma unroll
         for (int h = 0; h < HB; ++h) {
-            const float x = t[i][h] + sd[h];
-            t[i][h] = u[i] >= 0 ? (x >= 0.f ? x : a.slope * x) * kLog2e : -CUDART_INF_F;
+            const float y = leaky(t[i][h] + sd[h]);
+            t[i][h] = (FULL || u[i] >= 0) ? y : -CUDART_INF_F;
         }
 }
 
-template <int HB, int S, int MODE>
+// running (max, sum) of one head over a batch of logits
+template <int HB>
+__device__ __forceinline__ void online_update(const float (&t)[kSlotsInFlight][HB], float (&m)[HB], float (&l)[HB])
+{
+#pragma unroll
+    for (int h = 0; h < HB; ++h) {
+        float mx = m[h];                                               // t[0] is a real slot, so mx ends finite
+#pragma unroll
+        for (int i = 0; i < kSlotsInFlight; ++i) mx = fmaxf(mx, t[i][h]);
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < kSlotsInFlight; ++i) sum += ex2(t[i][h] - mx);                  // 2^-inf = 0
+        l[h] = l[h] * ex2(m[h] - mx) + sum;
+        m[h] = mx;
+    }
+}
+
+// One row (or hub segment) per S = LPS * SP lanes: SP slots are worked on side by side, and the heads
+// of a slot are spread over LPS lanes holding HB heads each (LPS * HB heads per round; more heads take
+// more rounds over the row).
+template <int HB, int LPS, int SP, int MODE>
 __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range& rg, int block_in_range)
 {
+    constexpr int S = LPS * SP;
     constexpr unsigned kFull = 0xffffffffu;
     const int tid = threadIdx.x;
     const int slot = block_in_range * (kBlock / S) + tid / S;
     const int sl = tid % S;
+    const int hb = sl % LPS;             // which block of HB heads of a slot
+    const int sp = sl / LPS;             // which of the SP slots of a step
     const bool active = slot < rg.item_count;
     int32_t row = 0, b = 0, e = 0;
     if (active) {
@@ -127,13 +178,16 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
         }
     }
     // every row of the warp fits one batch: the write pass reuses the logits of the first pass
-    const bool fits = MODE == kModeRows && __all_sync(kFull, e - b <= S * kSlotsInFlight);
+    const bool fits = MODE == kModeRows && __all_sync(kFull, e - b <= SP * kSlotsInFlight);
+    const Leaky leaky(a.slope);
 
-    for (int h0 = 0; h0 < a.heads; h0 += HB) {
+    for (int hh = 0; hh < a.heads; hh += LPS * HB) {
+        const int h0 = hh + hb * HB;
+        const bool head_ok = h0 < a.heads;
         float sd[HB];
 #pragma unroll
         for (int h = 0; h < HB; ++h) sd[h] = 0.f;
-        if (active) load_heads<HB>(a.s_dst + (int64_t)row * a.heads + h0, sd);
+        if (active && head_ok) load_heads<HB>(a.s_dst + (int64_t)row * a.heads + h0, sd);
         const float* ssrc = a.s_src + h0;
         float m[HB], inv[HB];
         float t[kSlotsInFlight][HB];
@@ -142,24 +196,27 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
             float l[HB];
 #pragma unroll
             for (int h = 0; h < HB; ++h) { m[h] = -CUDART_INF_F; l[h] = 0.f; }
-            for (int32_t k = b + sl; k < e; k += S * kSlotsInFlight) {
-                load_logits<HB, S>(a, ssrc, sd, k, e, t);
+            if (head_ok) {
+                int32_t u[kSlotsInFlight], un[kSlotsInFlight];
+                load_cols<SP>(a, b + sp, e, u);
+                for (int32_t kb = b; kb < e; kb += SP * kSlotsInFlight) {
+                    // the next batch's indices are on their way while this batch is gathered and reduced
+                    load_cols<SP>(a, kb + SP * kSlotsInFlight + sp, e, un);
+                    if (kb + SP * kSlotsInFlight <= e) {               // the same for all lanes of the row
+                        load_logits<HB, true>(a, leaky, ssrc, sd, u, t);
+                        online_update<HB>(t, m, l);
+                    } else if (u[0] >= 0) {
+                        load_logits<HB, false>(a, leaky, ssrc, sd, u, t);
+                        online_update<HB>(t, m, l);
+                    }
 #pragma unroll
-                for (int h = 0; h < HB; ++h) {
-                    float mx = m[h];                                   // t[0] is a real slot, so mx ends finite
-#pragma unroll
-                    for (int i = 0; i < kSlotsInFlight; ++i) mx = fmaxf(mx, t[i][h]);
-                    float sum = 0.f;
-#pragma unroll
-                    for (int i = 0; i < kSlotsInFlight; ++i) sum += exp2f(t[i][h] - mx);      // 2^-inf = 0
-                    l[h] = l[h] * rescale(m[h], mx) + sum;
-                    m[h] = mx;
+                    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = un[i];
                 }
             }
-            // butterfly over the S lanes of the row; both partners evaluate the same commutative expression
-            if constexpr (S > 1) {
+            // butterfly over the SP lanes that hold the same heads; both partners evaluate the same commutative expression
+            if constexpr (SP > 1) {
 #pragma unroll
-                for (int o = S / 2; o >= 1; o >>= 1)
+                for (int o = S / 2; o >= LPS; o >>= 1)
 #pragma unroll
                     for (int h = 0; h < HB; ++h) {
                         const float mo = __shfl_xor_sync(kFull, m[h], o);
@@ -169,55 +226,72 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
                         m[h] = mx;
                     }
             }
-            if (MODE == kModeHubStats) {
-                if (active && sl == 0) {
+            if constexpr (MODE == kModeHubStats) {
+                if (active && head_ok && sp == 0) {
 #pragma unroll
                     for (int h = 0; h < HB; ++h) a.seg_stats[(int64_t)slot * a.heads + h0 + h] = make_float2(m[h], l[h]);
                 }
-                continue;
             }
 #pragma unroll
             for (int h = 0; h < HB; ++h) inv[h] = 1.f / l[h];          // unused (inf) for an empty row
         } else {
 #pragma unroll
             for (int h = 0; h < HB; ++h) {
-                const float2 st = active ? a.seg_stats[(int64_t)slot * a.heads + h0 + h] : make_float2(0.f, 0.f);
+                const float2 st = (active && head_ok) ? a.seg_stats[(int64_t)slot * a.heads + h0 + h] : make_float2(0.f, 0.f);
                 m[h] = st.x;
                 inv[h] = st.y;
             }
         }
+        if (MODE == kModeHubStats || !head_ok) continue;
 
         if (fits) {
 #pragma unroll
             for (int i = 0; i < kSlotsInFlight; ++i) {
-                const int32_t k = b + sl + i * S;
+                const int32_t k = b + sp + i * SP;
                 if (k < e) {
                     float w[HB];
 #pragma unroll
-                    for (int h = 0; h < HB; ++h) w[h] = exp2f(t[i][h] - m[h]) * inv[h];
+                    for (int h = 0; h < HB; ++h) w[h] = ex2(t[i][h] - m[h]) * inv[h];
                     store_heads<HB>(a.alpha + (int64_t)k * a.heads + h0, w);
                 }
             }
         } else {
-            for (int32_t k = b + sl; k < e; k += S * kSlotsInFlight) {
-                load_logits<HB, S>(a, ssrc, sd, k, e, t);
+            int32_t u[kSlotsInFlight], un[kSlotsInFlight];
+            load_cols<SP>(a, b + sp, e, u);
+            for (int32_t kb = b; kb < e; kb += SP * kSlotsInFlight) {
+                const int32_t k = kb + sp;
+                load_cols<SP>(a, k + SP * kSlotsInFlight, e, un);
+                if (kb + SP * kSlotsInFlight <= e) {
+                    load_logits<HB, true>(a, leaky, ssrc, sd, u, t);
 #pragma unroll
-                for (int i = 0; i < kSlotsInFlight; ++i) {
-                    if (k + i * S < e) {
+                    for (int i = 0; i < kSlotsInFlight; ++i) {
                         float w[HB];
 #pragma unroll
-                        for (int h = 0; h < HB; ++h) w[h] = exp2f(t[i][h] - m[h]) * inv[h];
-                        store_heads<HB>(a.alpha + (int64_t)(k + i * S) * a.heads + h0, w);
+                        for (int h = 0; h < HB; ++h) w[h] = ex2(t[i][h] - m[h]) * inv[h];
+                        store_heads<HB>(a.alpha + (int64_t)(k + i * SP) * a.heads + h0, w);
+                    }
+                } else if (u[0] >= 0) {
+                    load_logits<HB, false>(a, leaky, ssrc, sd, u, t);
+#pragma unroll
+                    for (int i = 0; i < kSlotsInFlight; ++i) {
+                        if (u[i] >= 0) {
+                            float w[HB];
+#pragma unroll
+                            for (int h = 0; h < HB; ++h) w[h] = ex2(t[i][h] - m[h]) * inv[h];
+                            store_heads<HB>(a.alpha + (int64_t)(k + i * SP) * a.heads + h0, w);
+                        }
                     }
                 }
+#pragma unroll
+                for (int i = 0; i < kSlotsInFlight; ++i) u[i] = un[i];
             }
         }
     }
 }
 
 // All ordinary rows (stats and write in one go) and, in the same grid, the write pass of the hub segments.
-template <int HB>
-__global__ void __launch_bounds__(kBlock) edge_softmax_rows(const __grid_constant__ SoftmaxArgs a)
+template <int HB, int LPS>
+__global__ void __launch_bounds__(kBlock, GNNFD_SOFTMAX_MIN_BLOCKS) edge_softmax_rows(const __grid_constant__ SoftmaxArgs a)
 {
     const int rb = blockIdx.x;
     int r = 0;
@@ -226,22 +300,22 @@ __global__ void __launch_bounds__(kBlock) edge_softmax_rows(const __grid_constan
         if (i < a.n_ranges && rb >= a.range[i].first_block) r = i;
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
-    if (rg.hub) { softmax_items<HB, 32, kModeHubWrite>(a, rg, bir); return; }
+    if (rg.hub) { softmax_items<HB, LPS, 32 / LPS, kModeHubWrite>(a, rg, bir); return; }
     switch (rg.ep_log2) {
-        case 0: softmax_items<HB, 1, kModeRows>(a, rg, bir); break;
-        case 1: softmax_items<HB, 2, kModeRows>(a, rg, bir); break;
-        case 2: softmax_items<HB, 4, kModeRows>(a, rg, bir); break;
-        case 3: softmax_items<HB, 8, kModeRows>(a, rg, bir); break;
-        case 4: softmax_items<HB, 16, kModeRows>(a, rg, bir); break;
-        default: softmax_items<HB, 32, kModeRows>(a, rg, bir); break;
+        case 0: softmax_items<HB, LPS, 1, kModeRows>(a, rg, bir); break;
+        case 1: if constexpr (LPS * 2 <= 32) softmax_items<HB, LPS, 2, kModeRows>(a, rg, bir); break;
+        case 2: if constexpr (LPS * 4 <= 32) softmax_items<HB, LPS, 4, kModeRows>(a, rg, bir); break;
+        case 3: if constexpr (LPS * 8 <= 32) softmax_items<HB, LPS, 8, kModeRows>(a, rg, bir); break;
+        case 4: if constexpr (LPS * 16 <= 32) softmax_items<HB, LPS, 16, kModeRows>(a, rg, bir); break;
+        default: if constexpr (LPS == 1) softmax_items<HB, LPS, 32, kModeRows>(a, rg, bir); break;
     }
 }
 
 // (max, sum) of every hub segment; range 0 of the plan is the hub range
-template <int HB>
-__global__ void __launch_bounds__(kBlock) edge_softmax_hub_stats(const __grid_constant__ SoftmaxArgs a)
+template <int HB, int LPS>
+__global__ void __launch_bounds__(kBlock, GNNFD_SOFTMAX_MIN_BLOCKS) edge_softmax_hub_stats(const __grid_constant__ SoftmaxArgs a)
 {
-    softmax_items<HB, 32, kModeHubStats>(a, a.range[0], blockIdx.x);
+    softmax_items<HB, LPS, 32 / LPS, kModeHubStats>(a, a.range[0], blockIdx.x);
 }
 
 // One thread per (hub row, head): merges the segment results in ascending segment order and leaves the
@@ -268,17 +342,20 @@ static size_t softmax_scratch_bytes(const gnnfd_csr_t* csr, int32_t heads)
     return align_up((size_t)csr->n_segments * (size_t)heads * sizeof(float2), 256);
 }
 
-template <int HB>
-static int launch_softmax(const gnnfd_csr_t* csr, SoftmaxArgs& a, int64_t blocks, cudaStream_t s)
+template <int HB, int LPS>
+static int launch_softmax(const gnnfd_csr_t* csr, SoftmaxArgs& a, cudaStream_t s)
 {
+    const int64_t blocks = plan_ranges(csr, LPS, a.range, &a.n_ranges);
+    if (blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
+    if (blocks == 0) return GNNFD_OK;
     if (csr->n_segments > 0) {
         const unsigned hub_blocks = (unsigned)((csr->n_segments + kBlock / 32 - 1) / (kBlock / 32));
-        GNNFD_LAUNCH("edge_softmax_hub_stats", s, edge_softmax_hub_stats<HB>, hub_blocks, kBlock, 0, a);
+        GNNFD_LAUNCH("edge_softmax_hub_stats", s, (edge_softmax_hub_stats<HB, LPS>), hub_blocks, kBlock, 0, a);
         const int64_t pairs = (int64_t)a.n_hub * a.heads;
         GNNFD_LAUNCH("edge_softmax_hub_merge", s, edge_softmax_hub_merge, (unsigned)((pairs + kBlock - 1) / kBlock), kBlock,
                      0, a);
     }
-    GNNFD_LAUNCH("edge_softmax_rows", s, edge_softmax_rows<HB>, (unsigned)blocks, kBlock, 0, a);
+    GNNFD_LAUNCH("edge_softmax_rows", s, (edge_softmax_rows<HB, LPS>), (unsigned)blocks, kBlock, 0, a);
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
 }
@@ -310,16 +387,20 @@ int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float
     a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin; a.hub_seg_ptr = csr->hub_seg_ptr;
     a.s_src = d_s_src; a.s_dst = d_s_dst; a.alpha = d_alpha; a.seg_stats = static_cast<float2*>(d_scratch);
     a.slope = negative_slope; a.heads = heads; a.n_hub = (int32_t)csr->bin_count[4];
-    const int64_t blocks = plan_ranges(csr, 1, a.range, &a.n_ranges);
-    if (blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
-    if (blocks == 0) return GNNFD_OK;
 
-    // heads a lane handles per load: the widest of 8 / 4 / 2 / 1 that divides heads and keeps every access aligned
+    // heads per lane (HB) and lanes per slot (LPS): 16-byte accesses when heads is a multiple of 4 and the
+    // pointers allow it, with the heads of a slot spread over up to 8 lanes so that a warp's accesses to
+    // alpha are contiguous; otherwise one lane per slot with 8- or 4-byte accesses
     const uintptr_t ptrs = (uintptr_t)d_s_src | (uintptr_t)d_s_dst | (uintptr_t)d_alpha;
-    if (heads % 8 == 0 && ptrs % 16 == 0) return launch_softmax<8>(csr, a, blocks, s);
-    if (heads % 4 == 0 && ptrs % 16 == 0) return launch_softmax<4>(csr, a, blocks, s);
-    if (heads % 2 == 0 && ptrs % 8 == 0) return launch_softmax<2>(csr, a, blocks, s);
-    return launch_softmax<1>(csr, a, blocks, s);
+    if (heads % 4 == 0 && ptrs % 16 == 0) {
+        const int blocks4 = heads / 4;
+        if (blocks4 % 8 == 0) return launch_softmax<4, 8>(csr, a, s);
+        if (blocks4 % 4 == 0) return launch_softmax<4, 4>(csr, a, s);
+        if (blocks4 % 2 == 0) return launch_softmax<4, 2>(csr, a, s);
+        return launch_softmax<4, 1>(csr, a, s);
+    }
+    if (heads % 2 == 0 && ptrs % 8 == 0) return launch_softmax<2, 1>(csr, a, s);
+    return launch_softmax<1, 1>(csr, a, s);
 }
 
 }  // extern "C"
