@@ -198,7 +198,7 @@ def run_reference(args):
     import oracle as orc
     w = make_workload(args.workload, args.seed)
     threads = orc.max_threads()
-    rows, src, dst = oracle_sample(w, args.cpu_rows)
+    rows, src, dst = oracle_sample(w, args.cpu_rows or 16384)
     for _ in range(args.warmup):
         oracle_step(w, rows, src, dst, threads)
     t0 = time.perf_counter()
@@ -430,7 +430,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             import oracle as orc
             threads = orc.max_threads()
-            rows, s_src, s_dst = oracle_sample(w, args.cpu_rows)
+            rows, s_src, s_dst = oracle_sample(w, args.cpu_rows or 98304)
             t0 = time.perf_counter()
             units = oracle_step(w, rows, s_src, s_dst, threads)
             dt = time.perf_counter() - t0
@@ -451,7 +451,9 @@ def main():
     ap.add_argument("--chunk-width", type=int, default=0, help="0 = the workload's default")
     ap.add_argument("--sweep", type=int, nargs="*", default=[], help="extra chunk widths to time (aggregation only)")
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--cpu-rows", type=int, default=16384, help="destination rows in the CPU-oracle sample")
+    ap.add_argument("--cpu-rows", type=int, default=0,
+                    help="destination rows in the CPU-oracle sample (0: 16384 per step of --impl reference, "
+                         "98304 for the one cpu_baseline step of the CUDA arm)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

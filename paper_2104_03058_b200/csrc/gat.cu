@@ -7,6 +7,8 @@
 // are merged by the usual log-sum-exp rule in a fixed order.
 #include <math_constants.h>
 
+#include <type_traits>
+
 #include "schedule.cuh"
 #include "vec.cuh"
 
@@ -34,12 +36,21 @@ struct GatArgs {
 __device__ __forceinline__ float widen(float x) { return x; }
 __device__ __forceinline__ float widen(__nv_bfloat16 x) { return __bfloat162float(x); }
 
-__device__ __forceinline__ float leaky(float x, float slope) { return x >= 0.f ? x : slope * x; }
 
-// weight of a partial result with running maximum m when merged under the maximum m_new
+constexpr float kLog2e = 1.4426950408889634f;
+
+// 2^x by the hardware approximation (2 ulp; results below 2^-126 become 0, 2^-inf = 0)
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// weight of a partial result with running maximum m (a base-2 logit) when merged under the maximum m_new
 __device__ __forceinline__ float merge_scale(float m, float m_new)
 {
-    return m == -CUDART_INF_F ? 0.f : expf(m - m_new);
+    return m == -CUDART_INF_F ? 0.f : exp2f(m - m_new);
 }
 
 // ------------------------------------------------------------------ scores
@@ -118,6 +129,9 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
     }
     const float sd = active ? a.s_dst[(int64_t)row * a.heads + h] : 0.f;
     const float* ssrc = a.s_src + h;
+    // logits are kept in base 2: LeakyReLU(x) * log2 e = c1 * x + c2 * |x|
+    const float c1 = 0.5f * kLog2e * (1.f + a.slope), c2 = 0.5f * kLog2e * (1.f - a.slope);
+    auto leaky2 = [c1, c2](float x) { return fmaf(fabsf(x), c2, x * c1); };
     const uint32_t ld = (uint32_t)a.ldz;
     const uint32_t heads = (uint32_t)a.heads;
 
@@ -148,50 +162,58 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
 #pragma unroll
         for (int r = 0; r < R; ++r) stage_col[buf][warp][r * 32 + lane] = ucur[r];
         __syncwarp();
+        // one group of UB entries: gathers issued together, then one update of the running softmax
+        auto steps = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll
-        for (int s0 = 0; s0 < SPB; s0 += UB) {
-            Vec<T, VECN> v[UB][VPL];
-            float lg[UB];
-            bool valid[UB];
+            for (int s0 = 0; s0 < SPB; s0 += UB) {
+                Vec<T, VECN> v[UB][VPL];
+                float lg[UB];
+                bool valid[UB];
 #pragma unroll
-            for (int i = 0; i < UB; ++i) {
-                const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
-                valid[i] = u >= 0;
-                const uint32_t uu = (uint32_t)max(u, 0);
-                lg[i] = valid[i] ? __ldg(ssrc + (size_t)uu * heads) : 0.f;
-                const size_t off = (size_t)uu * ld;
+                for (int i = 0; i < UB; ++i) {
+                    const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
+                    const int32_t u = stage_col[buf][warp][r * 32 + seg + t * EP + g];
+                    valid[i] = FULL || u >= 0;
+                    const uint32_t uu = FULL ? (uint32_t)u : (uint32_t)max(u, 0);
+                    lg[i] = valid[i] ? __ldg(ssrc + (size_t)uu * heads) : 0.f;
+                    const size_t off = (size_t)uu * ld;
 #pragma unroll
-                for (int q = 0; q < VPL; ++q) {
-                    if (valid[i]) v[i][q].load(zq[q] + off);
-                    else v[i][q].zero();
+                    for (int q = 0; q < VPL; ++q) {
+                        if (valid[i]) v[i][q].load(zq[q] + off);
+                        else v[i][q].zero();
+                    }
+                }
+                float mx = m;
+#pragma unroll
+                for (int i = 0; i < UB; ++i) {
+                    lg[i] = leaky2(lg[i] + sd);
+                    if (valid[i]) mx = fmaxf(mx, lg[i]);
+                }
+                if (FULL || mx != -CUDART_INF_F) {      // a group with no entry at all leaves the state alone
+                    const float rescale = ex2(m - mx);  // 2^-inf = 0 on the first group
+                    m = mx;
+                    l *= rescale;
+#pragma unroll
+                    for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                        for (int i = 0; i < VECN; ++i) acc[q][i] *= rescale;
+                }
+#pragma unroll
+                for (int i = 0; i < UB; ++i) {
+                    // hardware 2^x: the argument is <= 0 and its error (about 2 ulp + |x| * 2^-23 relative) stays
+                    // two orders below the 1e-5 bound on the weighted sum
+                    const float p = valid[i] ? ex2(lg[i] - m) : 0.f;
+                    l += p;
+#pragma unroll
+                    for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                        for (int k = 0; k < VECN; ++k) acc[q][k] = fmaf(p, v[i][q].get(k), acc[q][k]);
                 }
             }
-            float mx = m;
-#pragma unroll
-            for (int i = 0; i < UB; ++i) {
-                lg[i] = leaky(lg[i] + sd, a.slope);
-                if (valid[i]) mx = fmaxf(mx, lg[i]);
-            }
-            const float rescale = merge_scale(m, mx);
-            m = mx;
-            l *= rescale;
-#pragma unroll
-            for (int q = 0; q < VPL; ++q)
-#pragma unroll
-                for (int i = 0; i < VECN; ++i) acc[q][i] *= rescale;
-#pragma unroll
-            for (int i = 0; i < UB; ++i) {
-                // fast exponential: the argument is <= 0 and its error (about 2 ulp + |x| * 2^-23 relative) stays
-                // two orders below the 1e-5 bound on the weighted sum; the merges below use expf
-                const float p = valid[i] ? __expf(lg[i] - m) : 0.f;
-                l += p;
-#pragma unroll
-                for (int q = 0; q < VPL; ++q)
-#pragma unroll
-                    for (int k = 0; k < VECN; ++k) acc[q][k] = fmaf(p, v[i][q].get(k), acc[q][k]);
-            }
-        }
+        };
+        if (__all_sync(kFull, kb + EPB <= e)) steps(std::true_type{});
+        else steps(std::false_type{});
 #pragma unroll
         for (int r = 0; r < R; ++r) ucur[r] = unext[r];
     }
