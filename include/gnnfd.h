@@ -212,6 +212,25 @@ int gnnfd_edge_softmax_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, si
 int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float* d_s_dst, int32_t heads,
                        float negative_slope, float* d_alpha, void* d_scratch, size_t scratch_bytes, void* stream);
 
+/* ------------------------------------------------------------------ Combination ahead of aggregation
+ *
+ * z[v, j] = sum_k x[v, k] * w_t[j, k]: the dense transform of a layer, applied to the input features
+ * before the aggregation so that the aggregation runs on the f_out transformed columns (Section III of
+ * the paper: the Combination phase is executed ahead of Aggregation; Algorithm 1 then decomposes the
+ * transformed features).  Not part of the aggregation path proper; offered so that a whole layer stays
+ * on the device.
+ *
+ * d_x [n, ldx] fp32, d_w_t [f_out, ldw] fp32 (the weight matrix transposed: one row per output column),
+ * d_z [n, ldz] fp32.  The product runs on the tensor cores: both operands are read as tf32 (the low 13
+ * mantissa bits of each fp32 value are ignored), products are exact, sums are fp32, so
+ * |z - exact| <= 2^-9 * sum_k |x[v,k] * w_t[j,k]| plus fp32 summation error.
+ * d_x and d_w_t must be 16-byte aligned with ldx and ldw multiples of 4 (GNNFD_UNSUPPORTED otherwise);
+ * d_z has no alignment rule.  d_status (may be NULL): one int32 the caller has set to 0; it becomes 1 if a
+ * block gave up waiting for its own copies or matrix instructions (each wait is limited to one second),
+ * in which case d_z is incomplete.  The call only enqueues work. */
+int gnnfd_combine(int64_t n, const float* d_x, int64_t ldx, int32_t f_in, const float* d_w_t, int64_t ldw,
+                  int32_t f_out, float* d_z, int64_t ldz, int32_t* d_status, void* stream);
+
 /* ------------------------------------------------------------------ diagnostics */
 
 const char* gnnfd_status_string(int status);

@@ -179,5 +179,19 @@ def aggregate_gat(row_ptr, col_idx, z, a_src, a_dst, heads: int, dim: int, slope
     return out, ab
 
 
+def combine(x: np.ndarray, w_t: np.ndarray, tf32: bool = False):
+    """Combination ahead of aggregation (Section III): z = x @ w_t.T in float64, and sum_k |x w| beside it.
+    With ``tf32`` both operands are first cut to the 10 explicit mantissa bits a tf32 operand keeps (the
+    low 13 bits of the fp32 pattern are dropped), which is what a tf32 tensor-core product computes
+    exactly apart from the order of its fp32 additions."""
+    x = np.ascontiguousarray(x, np.float32)
+    w_t = np.ascontiguousarray(w_t, np.float32)
+    if tf32:
+        x = (x.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+        w_t = (w_t.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+    x64, w64 = x.astype(np.float64), w_t.astype(np.float64)
+    return x64 @ w64.T, np.abs(x64) @ np.abs(w64).T
+
+
 def max_threads() -> int:
     return int(_load().orc_max_threads())

@@ -1,0 +1,339 @@
+// Combination ahead of aggregation (Section III of the paper runs the dense transform first, so that
+// the aggregation works on the narrower transformed features): z[n, f_out] = x[n, f_in] * W, W given
+// transposed as w_t[f_out, f_in].
+//
+// This is a dense contraction, so it runs on the tensor cores: tcgen05.mma with tf32 operands read
+// from shared memory, fp32 accumulation in tensor memory.  With f_out of 8 - 256 the product is bound
+// by streaming x from HBM once (f_in * 4 bytes per row against 2 * f_in * f_out flops), which the
+// fp32 ALUs could not keep up with.
+//
+// One block per 128 rows of x and per tile of up to 256 output columns.  Roles inside a block of four
+// warps: one lane of warp 0 issues the TMA loads (x tile 128 x 32 floats, w_t tile N x 32 floats, both
+// with the 128-byte swizzle) into a ring of stages, one lane of warp 1 issues four K = 8 MMAs per
+// stage and commits them to the stage's "empty" barrier, warp 2 owns the tensor-memory allocation;
+// after the last commit all four warps read the accumulator (warp w owns lanes 32 w .. 32 w + 31,
+// i.e. one output row per thread) and store it.  Rows past n and columns past f_in are filled with
+// zeros by the TMA unit, so ragged sizes need no special tiles.
+//
+// Every wait on a barrier is bounded: when a limit runs out the block records an error in the
+// caller's status word, drains the copies it has in flight (again bounded), frees its tensor memory
+// and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace gnnfd {
+
+constexpr int kCombineThreads = 128;
+constexpr int kTileM = 128;                 // rows of x per block (the MMA's M)
+constexpr int kTileK = 32;                  // floats per stage row: one 128-byte swizzle span
+constexpr int kMmaK = 8;                    // K of one tf32 MMA (32 bytes)
+constexpr int kMaxTileN = 256;
+constexpr uint64_t kWaitNs = 1000000000ull; // one second on one barrier before the block gives up
+constexpr int kSmemBudget = 100 * 1024;     // per block, so that two blocks share an SM
+constexpr int kMaxStages = 4;
+
+struct CombineArgs {
+    float* z;
+    int64_t ldz;
+    int32_t n, f_in, f_out, tile_n, stages, tmem_cols;
+    int32_t* status;        // set to 1 when a wait ran out (may be null)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ uint64_t now_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ bool mbar_test(uint32_t addr, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// true once the phase with the given parity has completed; gives up after kWaitNs
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    const uint32_t addr = smem_u32(bar);
+    if (mbar_test(addr, parity)) return true;
+    const uint64_t t0 = now_ns();
+    while (!mbar_test(addr, parity))
+        if (now_ns() - t0 > kWaitNs) return false;
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int32_t x, int32_t y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        :
+        : "r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+
+// Shared-memory operand descriptor of a K-major tile whose rows are 128 bytes, stored with the 128-byte
+// swizzle: groups of 8 rows are 1024 bytes apart; descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr)
+{
+    uint64_t d = (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;                    // leading-dimension offset: not used by swizzled K-major tiles
+    d |= (uint64_t)(1024 >> 4) << 32;          // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                    // descriptor version
+    d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulator, tf32 A and B, both K-major, M = 128, N = tile_n.
+__device__ __forceinline__ uint32_t instr_desc(int tile_n)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+        "}"
+        :
+        : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// arrives on the barrier once every MMA issued so far by this thread has finished
+__device__ __forceinline__ void mma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(kCombineThreads)
+combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CombineArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    // the dynamic buffer is aligned to 1024 bytes by hand (the swizzle pattern repeats every 1024 bytes)
+    unsigned char* tiles = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const uint32_t a_bytes = kTileM * kTileK * 4;
+    const uint32_t b_bytes = (uint32_t)a.tile_n * kTileK * 4;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = blockIdx.x * kTileM;
+    const int col0 = blockIdx.y * a.tile_n;
+    const int k_blocks = (a.f_in + kTileK - 1) / kTileK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < a.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"((uint32_t)a.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0 && lane == 0) {
+        // producer: fills stage kb % stages once the MMAs that read its previous contents have finished
+        int issued = 0;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % a.stages;
+            if (kb >= a.stages) ok = mbar_wait(&empty_bar[s], ((kb / a.stages) - 1) & 1);
+            if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
+            unsigned char* stage = tiles + (size_t)s * stage_bytes;
+            mbar_expect_tx(&full_bar[s], stage_bytes);
+            tma_load_2d(stage, &map_x, &full_bar[s], kb * kTileK, row0);
+            tma_load_2d(stage + a_bytes, &map_w, &full_bar[s], kb * kTileK, col0);
+            issued = kb + 1;
+        }
+        if (!ok) {
+            *(volatile int*)&abort_flag = 1;
+            // the copies already issued must land before the block's shared memory is given back
+            const int first = issued > a.stages ? issued - a.stages : 0;
+            for (int kb = first; kb < issued; ++kb) mbar_wait(&full_bar[kb % a.stages], (kb / a.stages) & 1);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // MMA issuer
+        const uint32_t idesc = instr_desc(a.tile_n);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % a.stages;
+            ok = mbar_wait(&full_bar[s], (kb / a.stages) & 1);
+            if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+            const uint32_t b_addr = a_addr + a_bytes;
+#pragma unroll
+            for (int k = 0; k < kTileK / kMmaK; ++k) {
+                // inside the 128-byte swizzle span the next K = 8 slice starts 32 bytes further on
+                const uint64_t da = operand_desc(a_addr + k * kMmaK * 4);
+                const uint64_t db = operand_desc(b_addr + k * kMmaK * 4);
+                mma_tf32(tmem_base, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            mma_commit(&empty_bar[s]);
+        }
+        if (ok) mma_commit(&accum_bar);
+        else *(volatile int*)&abort_flag = 1;
+    }
+    __syncwarp();
+
+    // epilogue: thread t of warp w holds row 32 w + t of the tile
+    bool ok = mbar_wait(&accum_bar, 0) && !*(volatile int*)&abort_flag;
+    // on an abort the accumulator barrier never completes: all lanes of all warps agree through the flag
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int row = row0 + warp * 32 + lane;
+        float* zrow = a.z + (int64_t)row * a.ldz + col0;
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(a.z) | (uintptr_t)(a.ldz * 4)) & 15u) == 0;
+        const int col_end = min(a.f_out, col0 + a.tile_n);
+        for (int c = 0; c < a.tile_n; c += 32) {
+            uint32_t r[32];
+            tmem_load_32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (row < a.n) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const int col = col0 + c + j;
+                    if (vec_ok && col + 4 <= col_end) {
+                        __stcs(reinterpret_cast<float4*>(zrow + c + j),
+                               make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                           __uint_as_float(r[j + 3])));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (col + i < col_end) zrow[c + j + i] = __uint_as_float(r[j + i]);
+                    }
+                }
+            }
+        }
+    } else if (threadIdx.x == 0 && a.status) {
+        atomicExch(a.status, 1);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// tensor map of a row-major fp32 matrix [rows, ld] of which `cols` columns are valid, box = box_rows x 32 floats
+static bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace gnnfd
+
+extern "C" int gnnfd_combine(int64_t n, const float* d_x, int64_t ldx, int32_t f_in, const float* d_w_t, int64_t ldw,
+                             int32_t f_out, float* d_z, int64_t ldz, int32_t* d_status, void* stream)
+{
+    using namespace gnnfd;
+    if (n <= 0 || !d_x || !d_w_t || !d_z || f_in <= 0 || f_out <= 0 || ldx < f_in || ldw < f_in || ldz < f_out)
+        return GNNFD_INVALID_ARG;
+    if (n > 0x7fffffffll - kTileM) return GNNFD_TOO_LARGE;
+    // the TMA unit wants 16-byte aligned bases and row pitches
+    if (((uintptr_t)d_x | (uintptr_t)d_w_t) % 16 != 0 || (ldx * 4) % 16 != 0 || (ldw * 4) % 16 != 0) return GNNFD_UNSUPPORTED;
+
+    CombineArgs a;
+    a.z = d_z; a.ldz = ldz; a.n = (int32_t)n; a.f_in = f_in; a.f_out = f_out; a.status = d_status;
+    // output columns per block: all of them up to 256, rounded up to the MMA's N granularity of 16
+    const int n_col_tiles = (f_out + kMaxTileN - 1) / kMaxTileN;
+    const int per_tile = (f_out + n_col_tiles - 1) / n_col_tiles;
+    a.tile_n = (per_tile + 15) / 16 * 16;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < a.tile_n) a.tmem_cols <<= 1;
+    const int stage_bytes = (kTileM + a.tile_n) * kTileK * 4;
+    a.stages = kSmemBudget / stage_bytes;
+    if (a.stages > kMaxStages) a.stages = kMaxStages;
+    if (a.stages < 2) return GNNFD_UNSUPPORTED;
+    const size_t smem = (size_t)a.stages * stage_bytes + 1024;
+
+    CUtensorMap map_x, map_w;
+    if (!make_map(&map_x, d_x, n, f_in, ldx, kTileM) || !make_map(&map_w, d_w_t, f_out, f_in, ldw, a.tile_n)) {
+        set_cuda_error(cudaErrorInvalidValue);
+        return GNNFD_CUDA_ERROR;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const dim3 grid((unsigned)((n + kTileM - 1) / kTileM), (unsigned)((f_out + a.tile_n - 1) / a.tile_n));
+    GNNFD_LAUNCH("combine_tf32", s, combine_tf32, grid, kCombineThreads, smem, map_x, map_w, a);
+    GNNFD_CUDA_CHECK(cudaGetLastError());
+    return GNNFD_OK;
+}

@@ -392,3 +392,41 @@ def test_leading_dimension_padding_is_ignored():
     a, _ = orc.aggregate("sage", row_ptr, col, x, 6, 4)
     b, _ = orc.aggregate("sage", row_ptr, col, np.ascontiguousarray(x[:, :6]), 6, 4)
     np.testing.assert_array_equal(a, b)
+
+
+# ------------------------------------------------------------------ Combination (dense transform ahead of aggregation)
+
+def test_combine_against_triple_loop_and_closed_forms():
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((7, 5)).astype(np.float32)
+    w_t = rng.standard_normal((3, 5)).astype(np.float32)
+    z, scale = orc.combine(x, w_t)
+    for v in range(7):
+        for j in range(3):
+            acc = sum(float(x[v, k]) * float(w_t[j, k]) for k in range(5))
+            assert abs(z[v, j] - acc) <= 1e-12 * (1 + abs(acc))
+            assert abs(scale[v, j] - sum(abs(float(x[v, k]) * float(w_t[j, k])) for k in range(5))) <= 1e-12 * scale[v, j]
+    # a transposed weight matrix must fail: w_t is [f_out, f_in], so x @ w_t.T, never x @ w_t
+    sq = rng.standard_normal((5, 5)).astype(np.float32)
+    assert not np.allclose(orc.combine(x, sq)[0], x.astype(np.float64) @ sq.astype(np.float64))
+    # identity weights return x; all-ones weights return the row sums
+    assert np.array_equal(orc.combine(x, np.eye(5, dtype=np.float32))[0], x.astype(np.float64))
+    np.testing.assert_allclose(orc.combine(x, np.ones((2, 5), np.float32))[0],
+                               np.repeat(x.astype(np.float64).sum(1)[:, None], 2, 1), rtol=1e-13)
+
+
+def test_combine_tf32_reading_cuts_thirteen_mantissa_bits():
+    one = np.float32(1.0)
+    ulp_tf32 = np.float32(2.0 ** -10)
+    x = np.array([[one + np.float32(2.0 ** -11), one + ulp_tf32, -(one + np.float32(2.0 ** -11)) - np.float32(2.0 ** -12)]],
+                 np.float32)
+    z, _ = orc.combine(x, np.eye(3, dtype=np.float32), tf32=True)
+    # below the last kept bit: dropped (towards zero, for either sign); the last kept bit itself stays
+    assert z[0, 0] == 1.0 and z[0, 1] == float(one + ulp_tf32) and z[0, 2] == -1.0
+    # the cut never moves a value by more than 2^-10 relative, so a product by less than 2^-9
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal((40, 30)).astype(np.float32)
+    b = rng.standard_normal((20, 30)).astype(np.float32)
+    exact, scale = orc.combine(a, b)
+    cut, _ = orc.combine(a, b, tf32=True)
+    assert (np.abs(cut - exact) <= 2.0 ** -9 * scale).all() and np.abs(cut - exact).max() > 0
