@@ -375,6 +375,26 @@ def run_ours(args):
         torch.cuda.synchronize()
         softmax_ms = a0.elapsed_time(a1) / reps
 
+    combine_ms = None
+    if not bf16 and args.combine_out > 0:
+        # the dense transform a layer runs ahead of its aggregation (Section III), timed alone: x [n, f] -> [n, combine_out]
+        w_t = (torch.randn((args.combine_out, w.ld), device=device) * 0.05)
+        z = torch.empty((w.n, args.combine_out), device=device)
+        status = torch.zeros(1, dtype=torch.int32, device=device)
+        for _ in range(3):
+            g.combine(d_x[:, :w.f], w_t[:, :w.f], out=z, status=status)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(20):
+            g.combine(d_x[:, :w.f], w_t[:, :w.f], out=z, status=status)
+        a1.record()
+        torch.cuda.synchronize()
+        if int(status.item()) != 0:
+            raise SystemExit("gnnfd_combine reported a timed-out wait")
+        combine_ms = a0.elapsed_time(a1) / 20
+        del z, w_t
+
     ms, total_units = sharding.reduce_job_timing(ms, float(units_per_step), device=device)
     ms_e2e, _ = sharding.reduce_job_timing(ms_e2e, 0.0, device=device)
 
@@ -427,6 +447,14 @@ def run_ours(args):
             result["edge_softmax_only"] = {"ms": softmax_ms, "alpha_GBs_written": nnz * w.heads * 4 / (softmax_ms * 1e-3) / 1e9,
                                            "hbm_bytes": sm_bytes, "hbm_GBs": sm_bytes / (softmax_ms * 1e-3) / 1e9,
                                            "frac_of_hbm_peak": sm_bytes / (softmax_ms * 1e-3) / 1e9 / peak}
+        if combine_ms is not None:
+            cb_bytes = 4 * (w.n * w.f + args.combine_out * w.f + w.n * args.combine_out)
+            result["combine_only"] = {
+                "kernel": "combine_tf32", "shape": "[%d, %d] x [%d, %d]" % (w.n, w.f, w.f, args.combine_out),
+                "ms": combine_ms, "bound": "hbm", "hbm_bytes": cb_bytes,
+                "achieved_GBs": cb_bytes / (combine_ms * 1e-3) / 1e9,
+                "frac_of_hbm_peak": cb_bytes / (combine_ms * 1e-3) / 1e9 / peak,
+                "tf32_TFLOPs": 2.0 * w.n * w.f * args.combine_out / (combine_ms * 1e-3) / 1e12}
         if world == 1 and not args.no_cpu_baseline:
             import oracle as orc
             threads = orc.max_threads()
@@ -450,6 +478,8 @@ def main():
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="config4")
     ap.add_argument("--chunk-width", type=int, default=0, help="0 = the workload's default")
     ap.add_argument("--sweep", type=int, nargs="*", default=[], help="extra chunk widths to time (aggregation only)")
+    ap.add_argument("--combine-out", type=int, default=64,
+                    help="output width of the dense transform timed beside the step (0: skip; fp32 workloads only)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-rows", type=int, default=0,
                     help="destination rows in the CPU-oracle sample (0: 16384 per step of --impl reference, "
