@@ -220,16 +220,20 @@ int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float
  * transformed features).  Not part of the aggregation path proper; offered so that a whole layer stays
  * on the device.
  *
- * d_x [n, ldx] fp32, d_w_t [f_out, ldw] fp32 (the weight matrix transposed: one row per output column),
- * d_z [n, ldz] fp32.  The product runs on the tensor cores: both operands are read as tf32 (the low 13
- * mantissa bits of each fp32 value are ignored), products are exact, sums are fp32, so
- * |z - exact| <= 2^-9 * sum_k |x[v,k] * w_t[j,k]| plus fp32 summation error.
- * d_x and d_w_t must be 16-byte aligned with ldx and ldw multiples of 4 (GNNFD_UNSUPPORTED otherwise);
- * d_z has no alignment rule.  d_status (may be NULL): one int32 the caller has set to 0; it becomes 1 if a
- * block gave up waiting for its own copies or matrix instructions (each wait is limited to one second),
- * in which case d_z is incomplete.  The call only enqueues work. */
-int gnnfd_combine(int64_t n, const float* d_x, int64_t ldx, int32_t f_in, const float* d_w_t, int64_t ldw,
-                  int32_t f_out, float* d_z, int64_t ldz, int32_t* d_status, void* stream);
+ * d_x [n, ldx] and d_w_t [f_out, ldw] (the weight matrix transposed: one row per output column) both of
+ * type xdt; d_z [n, ldz] of type zdt.  The product runs on the tensor cores with fp32 sums:
+ *   xdt = GNNFD_F32 : both operands are read as tf32 (the low 13 mantissa bits of each fp32 value are
+ *                     ignored), products are exact, so |z - exact| <= 2^-9 * sum_k |x[v,k] * w_t[j,k]|
+ *                     plus fp32 summation error;
+ *   xdt = GNNFD_BF16: operands are used as they are, products are exact in fp32.
+ * zdt = GNNFD_BF16 rounds the fp32 result to nearest even.
+ * d_x and d_w_t must be 16-byte aligned with row pitches that are multiples of 16 bytes
+ * (GNNFD_UNSUPPORTED otherwise); d_z has no alignment rule.  d_status (may be NULL): one int32 the caller
+ * has set to 0; it becomes 1 if a block gave up waiting for its own copies or matrix instructions (each
+ * wait is limited to one second), in which case d_z is incomplete.  The call only enqueues work. */
+int gnnfd_combine(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t,
+                  int64_t ldw, int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int32_t* d_status,
+                  void* stream);
 
 /* ------------------------------------------------------------------ diagnostics */
 

@@ -63,7 +63,7 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_aggregate_gat.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32, vp, sz, vp]
         L.gnnfd_edge_softmax_workspace_bytes.argtypes = [vp, i32, pp(sz)]
         L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp, sz, vp]
-        L.gnnfd_combine.argtypes = [i64, vp, i64, i32, vp, i64, i32, vp, i64, vp, vp]
+        L.gnnfd_combine.argtypes = [i64, vp, i64, i32, i32, vp, i64, i32, vp, i64, i32, vp, vp]
         L.gnnfd_status_string.argtypes = [ctypes.c_int]
         L.gnnfd_status_string.restype = ctypes.c_char_p
         L.gnnfd_last_cuda_error.restype = ctypes.c_int
@@ -342,21 +342,22 @@ def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_sl
 
 
 def combine(x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, out: torch.Tensor | None = None,
-            status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """gnnfd_combine: z = x[:, :f_in] @ w_t[:, :f_in].T on the tensor cores (tf32 operands, fp32 sums).
-    ``status`` is an int32 tensor of one element that the kernel sets to 1 if a block gave up waiting."""
+            out_dtype=None, status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """gnnfd_combine: z = x[:, :f_in] @ w_t[:, :f_in].T on the tensor cores (tf32 operands for float32
+    inputs, bf16 operands for bfloat16 inputs; fp32 sums).  ``status`` is an int32 tensor of one element
+    that the kernel sets to 1 if a block gave up waiting."""
     f_in = w_t.shape[1] if f_in is None else f_in
     f_out = w_t.shape[0]
-    if x.dtype != torch.float32 or w_t.dtype != torch.float32:
-        raise TypeError("combine takes float32 matrices")
+    if x.dtype != w_t.dtype:
+        raise TypeError("x and w_t must have the same dtype")
     if out is None:
-        out = torch.empty((x.shape[0], f_out), dtype=torch.float32, device=x.device)
+        out = torch.empty((x.shape[0], f_out), dtype=out_dtype or torch.float32, device=x.device)
     xp, ldx = _matrix(x, f_in, "x")
     wp, ldw = _matrix(w_t, f_in, "w_t")
     op, ldo = _matrix(out, f_out, "out")
     sp = ctypes.c_void_p(status.data_ptr()) if status is not None else None
-    _check(lib().gnnfd_combine(x.shape[0], xp, ldx, f_in, wp, ldw, f_out, op, ldo, sp, _stream_ptr(stream)),
-           "gnnfd_combine")
+    _check(lib().gnnfd_combine(x.shape[0], xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, op, ldo, _dtype_code(out), sp,
+                               _stream_ptr(stream)), "gnnfd_combine")
     return out
 
 

@@ -2,14 +2,14 @@
 // the aggregation works on the narrower transformed features): z[n, f_out] = x[n, f_in] * W, W given
 // transposed as w_t[f_out, f_in].
 //
-// This is a dense contraction, so it runs on the tensor cores: tcgen05.mma with tf32 operands read
-// from shared memory, fp32 accumulation in tensor memory.  With f_out of 8 - 256 the product is bound
+// This is a dense contraction, so it runs on the tensor cores: tcgen05.mma with tf32 operands (fp32
+// inputs) or bf16 operands (bf16 inputs) read from shared memory, fp32 accumulation in tensor memory.  With f_out of 8 - 256 the product is bound
 // by streaming x from HBM once (f_in * 4 bytes per row against 2 * f_in * f_out flops), which the
 // fp32 ALUs could not keep up with.
 //
 // One block per 128 rows of x and per tile of up to 256 output columns.  Roles inside a block of four
-// warps: one lane of warp 0 issues the TMA loads (x tile 128 x 32 floats, w_t tile N x 32 floats, both
-// with the 128-byte swizzle) into a ring of stages, one lane of warp 1 issues four K = 8 MMAs per
+// warps: one lane of warp 0 issues the TMA loads (x tile 128 rows x 128 bytes, w_t tile N rows x 128 bytes,
+// both with the 128-byte swizzle) into a ring of stages, one lane of warp 1 issues four 32-byte-deep MMAs per
 // stage and commits them to the stage's "empty" barrier, warp 2 owns the tensor-memory allocation;
 // after the last commit all four warps read the accumulator (warp w owns lanes 32 w .. 32 w + 31,
 // i.e. one output row per thread) and store it.  Rows past n and columns past f_in are filled with
@@ -19,6 +19,7 @@
 // caller's status word, drains the copies it has in flight (again bounded), frees its tensor memory
 // and returns.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include "common.cuh"
 
@@ -26,17 +27,17 @@ namespace gnnfd {
 
 constexpr int kCombineThreads = 128;
 constexpr int kTileM = 128;                 // rows of x per block (the MMA's M)
-constexpr int kTileK = 32;                  // floats per stage row: one 128-byte swizzle span
-constexpr int kMmaK = 8;                    // K of one tf32 MMA (32 bytes)
+constexpr int kTileKBytes = 128;            // bytes per stage row: one 128-byte swizzle span (32 floats or 64 bf16)
+constexpr int kMmaKBytes = 32;              // depth of one MMA: K = 8 for tf32, K = 16 for bf16
 constexpr int kMaxTileN = 256;
 constexpr uint64_t kWaitNs = 1000000000ull; // one second on one barrier before the block gives up
 constexpr int kSmemBudget = 100 * 1024;     // per block, so that two blocks share an SM
 constexpr int kMaxStages = 4;
 
 struct CombineArgs {
-    float* z;
+    void* z;
     int64_t ldz;
-    int32_t n, f_in, f_out, tile_n, stages, tmem_cols;
+    int32_t n, f_in, f_out, tile_n, stages, tmem_cols, z_bf16;
     int32_t* status;        // set to 1 when a wait ran out (may be null)
 };
 
@@ -106,23 +107,39 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr)
     return d;
 }
 
-// Instruction descriptor: fp32 accumulator, tf32 A and B, both K-major, M = 128, N = tile_n.
+// Instruction descriptor: fp32 accumulator, A and B of one type (format 2 = tf32, 1 = bf16), both
+// K-major, M = 128, N = tile_n.
+template <bool BF16>
 __device__ __forceinline__ uint32_t instr_desc(int tile_n)
 {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    constexpr uint32_t fmt = BF16 ? 1u : 2u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
-__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+template <bool BF16>
+__device__ __forceinline__ void mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
-        "}"
-        :
-        : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if constexpr (BF16) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
 
 // arrives on the barrier once every MMA issued so far by this thread has finished
@@ -145,8 +162,9 @@ __device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
 }
 
+template <bool BF16>
 __global__ void __launch_bounds__(kCombineThreads)
-combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CombineArgs a)
+combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CombineArgs a)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
@@ -155,8 +173,9 @@ combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 
     // the dynamic buffer is aligned to 1024 bytes by hand (the swizzle pattern repeats every 1024 bytes)
     unsigned char* tiles = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const uint32_t a_bytes = kTileM * kTileK * 4;
-    const uint32_t b_bytes = (uint32_t)a.tile_n * kTileK * 4;
+    constexpr int kTileK = kTileKBytes / (BF16 ? 2 : 4);      // elements of K per stage
+    const uint32_t a_bytes = kTileM * kTileKBytes;
+    const uint32_t b_bytes = (uint32_t)a.tile_n * kTileKBytes;
     const uint32_t stage_bytes = a_bytes + b_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -203,7 +222,7 @@ combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         }
     } else if (warp == 1 && lane == 0) {
         // MMA issuer
-        const uint32_t idesc = instr_desc(a.tile_n);
+        const uint32_t idesc = instr_desc<BF16>(a.tile_n);
         bool ok = true;
         for (int kb = 0; kb < k_blocks && ok; ++kb) {
             const int s = kb % a.stages;
@@ -213,11 +232,11 @@ combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
             const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-            for (int k = 0; k < kTileK / kMmaK; ++k) {
-                // inside the 128-byte swizzle span the next K = 8 slice starts 32 bytes further on
-                const uint64_t da = operand_desc(a_addr + k * kMmaK * 4);
-                const uint64_t db = operand_desc(b_addr + k * kMmaK * 4);
-                mma_tf32(tmem_base, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kTileKBytes / kMmaKBytes; ++k) {
+                // inside the 128-byte swizzle span the next K slice starts 32 bytes further on
+                const uint64_t da = operand_desc(a_addr + k * kMmaKBytes);
+                const uint64_t db = operand_desc(b_addr + k * kMmaKBytes);
+                mma<BF16>(tmem_base, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             }
             mma_commit(&empty_bar[s]);
         }
@@ -233,25 +252,47 @@ combine_tf32(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     if (ok) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int row = row0 + warp * 32 + lane;
-        float* zrow = a.z + (int64_t)row * a.ldz + col0;
-        const bool vec_ok = ((reinterpret_cast<uintptr_t>(a.z) | (uintptr_t)(a.ldz * 4)) & 15u) == 0;
         const int col_end = min(a.f_out, col0 + a.tile_n);
+        const int zsize = a.z_bf16 ? 2 : 4;
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(a.z) | (uintptr_t)(a.ldz * zsize)) & 15u) == 0;
         for (int c = 0; c < a.tile_n; c += 32) {
             uint32_t r[32];
             tmem_load_32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (row < a.n) {
+            if (row >= a.n) continue;
+            if (a.z_bf16) {
+                __nv_bfloat16* zrow = static_cast<__nv_bfloat16*>(a.z) + (int64_t)row * a.ldz + col0 + c;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    const int col = col0 + c + j;
+                    if (vec_ok && col + 8 <= col_end) {
+                        uint4 v;
+                        uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * i]), __uint_as_float(r[j + 2 * i + 1]));
+                            pv[i] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        __stcs(reinterpret_cast<uint4*>(zrow + j), v);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (col + i < col_end) zrow[j + i] = __float2bfloat16_rn(__uint_as_float(r[j + i]));
+                    }
+                }
+            } else {
+                float* zrow = static_cast<float*>(a.z) + (int64_t)row * a.ldz + col0 + c;
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     const int col = col0 + c + j;
                     if (vec_ok && col + 4 <= col_end) {
-                        __stcs(reinterpret_cast<float4*>(zrow + c + j),
+                        __stcs(reinterpret_cast<float4*>(zrow + j),
                                make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
                                            __uint_as_float(r[j + 3])));
                     } else {
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            if (col + i < col_end) zrow[c + j + i] = __uint_as_float(r[j + i]);
+                            if (col + i < col_end) zrow[j + i] = __uint_as_float(r[j + i]);
                     }
                 }
             }
@@ -285,55 +326,67 @@ static EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// tensor map of a row-major fp32 matrix [rows, ld] of which `cols` columns are valid, box = box_rows x 32 floats
-static bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+// tensor map of a row-major matrix [rows, ld] of which `cols` columns are valid; box = box_rows x 128 bytes
+static bool make_map(CUtensorMap* map, const void* base, bool bf16, int64_t rows, int64_t cols, int64_t ld, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const int esize = bf16 ? 2 : 4;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * esize};
+    const cuuint32_t box[2] = {(cuuint32_t)(kTileKBytes / esize), (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims,
+              strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace gnnfd
 
-extern "C" int gnnfd_combine(int64_t n, const float* d_x, int64_t ldx, int32_t f_in, const float* d_w_t, int64_t ldw,
-                             int32_t f_out, float* d_z, int64_t ldz, int32_t* d_status, void* stream)
+extern "C" int gnnfd_combine(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t,
+                             int64_t ldw, int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int32_t* d_status,
+                             void* stream)
 {
     using namespace gnnfd;
     if (n <= 0 || !d_x || !d_w_t || !d_z || f_in <= 0 || f_out <= 0 || ldx < f_in || ldw < f_in || ldz < f_out)
         return GNNFD_INVALID_ARG;
+    if ((xdt != GNNFD_F32 && xdt != GNNFD_BF16) || (zdt != GNNFD_F32 && zdt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
     if (n > 0x7fffffffll - kTileM) return GNNFD_TOO_LARGE;
+    const bool bf16 = xdt == GNNFD_BF16;
+    const int esize = bf16 ? 2 : 4;
     // the TMA unit wants 16-byte aligned bases and row pitches
-    if (((uintptr_t)d_x | (uintptr_t)d_w_t) % 16 != 0 || (ldx * 4) % 16 != 0 || (ldw * 4) % 16 != 0) return GNNFD_UNSUPPORTED;
+    if (((uintptr_t)d_x | (uintptr_t)d_w_t) % 16 != 0 || (ldx * esize) % 16 != 0 || (ldw * esize) % 16 != 0)
+        return GNNFD_UNSUPPORTED;
 
     CombineArgs a;
     a.z = d_z; a.ldz = ldz; a.n = (int32_t)n; a.f_in = f_in; a.f_out = f_out; a.status = d_status;
+    a.z_bf16 = zdt == GNNFD_BF16;
     // output columns per block: all of them up to 256, rounded up to the MMA's N granularity of 16
     const int n_col_tiles = (f_out + kMaxTileN - 1) / kMaxTileN;
     const int per_tile = (f_out + n_col_tiles - 1) / n_col_tiles;
     a.tile_n = (per_tile + 15) / 16 * 16;
     a.tmem_cols = 32;
     while (a.tmem_cols < a.tile_n) a.tmem_cols <<= 1;
-    const int stage_bytes = (kTileM + a.tile_n) * kTileK * 4;
+    const int stage_bytes = (kTileM + a.tile_n) * kTileKBytes;
     a.stages = kSmemBudget / stage_bytes;
     if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return GNNFD_UNSUPPORTED;
     const size_t smem = (size_t)a.stages * stage_bytes + 1024;
 
     CUtensorMap map_x, map_w;
-    if (!make_map(&map_x, d_x, n, f_in, ldx, kTileM) || !make_map(&map_w, d_w_t, f_out, f_in, ldw, a.tile_n)) {
+    if (!make_map(&map_x, d_x, bf16, n, f_in, ldx, kTileM) || !make_map(&map_w, d_w_t, bf16, f_out, f_in, ldw, a.tile_n)) {
         set_cuda_error(cudaErrorInvalidValue);
         return GNNFD_CUDA_ERROR;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const dim3 grid((unsigned)((n + kTileM - 1) / kTileM), (unsigned)((f_out + a.tile_n - 1) / a.tile_n));
-    GNNFD_LAUNCH("combine_tf32", s, combine_tf32, grid, kCombineThreads, smem, map_x, map_w, a);
+    if (bf16) {
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_bf16", s, combine_mma<true>, grid, kCombineThreads, smem, map_x, map_w, a);
+    } else {
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_tf32", s, combine_mma<false>, grid, kCombineThreads, smem, map_x, map_w, a);
+    }
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
 }

@@ -95,3 +95,39 @@ def test_combine_then_aggregate_is_a_gcn_layer(g):
     want, _ = orc.aggregate("gcn", row_ptr, col, z_cut.astype(np.float32), f_out)
     bound, _ = orc.aggregate("gcn", row_ptr, col, z_scale.astype(np.float32), f_out)
     assert (np.abs(out - want) <= 2e-5 * bound + 2e-6).all()
+
+
+def _bf16(a):
+    """bf16 bit patterns (uint16), the same values widened to float32, and a torch bfloat16 device tensor"""
+    bits = gg.to_bf16_bits(a)
+    wide = (bits.astype(np.uint32) << 16).view(np.float32)
+    dev = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    return bits, wide, dev
+
+
+@pytest.mark.parametrize("n,f_in,ld,f_out", [(1000, 256, 256, 64), (333, 100, 104, 24), (130, 64, 64, 8), (260, 72, 72, 272)])
+def test_combine_bf16_operands(g, n, f_in, ld, f_out):
+    """bf16 inputs are used as they are: products are exact in fp32, so only the summation order differs
+    from the oracle run on the widened values."""
+    x = gg.features_f32(n, ld, dist="uniform", p0=-1.0, p1=1.0, seed=n)
+    w_t = gg.features_f32(f_out, ld, dist="normal", p0=0.0, p1=0.3, seed=n, stream=8)
+    _, xw, xd = _bf16(x)
+    _, ww, wd = _bf16(w_t)
+    exact, scale = orc.combine(xw[:, :f_in], ww[:, :f_in])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = g.combine(xd[:, :f_in], wd[:, :f_in], status=status).cpu().numpy().astype(np.float64)
+    assert int(status.item()) == 0
+    assert (np.abs(got - exact) <= 1e-5 * scale + 1e-6).all()
+    # bf16 output: the fp32 result rounded to nearest even (half an ulp = 2^-9 relative)
+    got16 = g.combine(xd[:, :f_in], wd[:, :f_in], out_dtype=torch.bfloat16).float().cpu().numpy().astype(np.float64)
+    assert (np.abs(got16 - exact) <= 2.0 ** -9 * np.abs(exact) + 1e-5 * scale + 1e-6).all()
+
+
+def test_combine_fp32_inputs_bf16_output(g):
+    n, f_in, f_out = 500, 96, 40
+    x = gg.features_f32(n, f_in, dist="normal", p0=0.0, p1=1.0, seed=21)
+    w_t = gg.features_f32(f_out, f_in, dist="normal", p0=0.0, p1=0.5, seed=21, stream=8)
+    cut, scale = orc.combine(x, w_t, tf32=True)
+    got = g.combine(torch.from_numpy(x).cuda(), torch.from_numpy(w_t).cuda(), out_dtype=torch.bfloat16)
+    got = got.float().cpu().numpy().astype(np.float64)
+    assert (np.abs(got - cut) <= 2.0 ** -9 * np.abs(cut) + 1e-5 * scale + 1e-6).all()
