@@ -118,9 +118,9 @@ def test_combine_bf16_operands(g, n, f_in, ld, f_out):
     got = g.combine(xd[:, :f_in], wd[:, :f_in], status=status).cpu().numpy().astype(np.float64)
     assert int(status.item()) == 0
     assert (np.abs(got - exact) <= 1e-5 * scale + 1e-6).all()
-    # bf16 output: the fp32 result rounded to nearest even (half an ulp = 2^-9 relative)
+    # bf16 output: the fp32 result rounded to nearest even (8 significant bits: half an ulp is at most 2^-8 relative)
     got16 = g.combine(xd[:, :f_in], wd[:, :f_in], out_dtype=torch.bfloat16).float().cpu().numpy().astype(np.float64)
-    assert (np.abs(got16 - exact) <= 2.0 ** -9 * np.abs(exact) + 1e-5 * scale + 1e-6).all()
+    assert (np.abs(got16 - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-5 * scale + 1e-6).all()
 
 
 def test_combine_fp32_inputs_bf16_output(g):
@@ -130,4 +130,4 @@ def test_combine_fp32_inputs_bf16_output(g):
     cut, scale = orc.combine(x, w_t, tf32=True)
     got = g.combine(torch.from_numpy(x).cuda(), torch.from_numpy(w_t).cuda(), out_dtype=torch.bfloat16)
     got = got.float().cpu().numpy().astype(np.float64)
-    assert (np.abs(got - cut) <= 2.0 ** -9 * np.abs(cut) + 1e-5 * scale + 1e-6).all()
+    assert (np.abs(got - cut) <= 2.0 ** -8 * np.abs(cut) + 1e-5 * scale + 1e-6).all()
