@@ -232,28 +232,95 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
 
 // ------------------------------------------------------------------ after the sort
 
-// flag[i] = 1 for the first of each run of equal keys among the kept candidates
-__global__ void __launch_bounds__(kThreads)
-flag_first_of_run(const u64* __restrict__ keys, int64_t m, int val_bits, const BuildCounts* __restrict__ counts,
-                  int32_t* __restrict__ flag)
+// Duplicate removal after the sort, in two sweeps with a scan of one count per tile between them: a
+// sorted candidate is kept when it is valid and its key differs from its predecessor's.  A thread
+// looks after kUniqueItems consecutive candidates, a block after kUniqueTile.
+constexpr int kUniqueItems = 8;
+constexpr int kUniqueTile = kThreads * kUniqueItems;
+
+// bit j of the result: candidate first + j is the first of a run of equal keys among the n_valid kept ones
+__device__ __forceinline__ uint32_t first_of_run_mask(const u64* __restrict__ keys, int64_t first, int64_t n_valid, int val_bits,
+                                                      u64 (&word)[kUniqueItems])
 {
-    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (i >= m) return;
-    flag[i] = (i < counts->n_valid && (i == 0 || (keys[i] >> val_bits) != (keys[i - 1] >> val_bits))) ? 1 : 0;
+    u64 prev = first > 0 && first <= n_valid ? (__ldg(keys + first - 1) >> val_bits) : 0ull;
+    uint32_t mask = 0;
+#pragma unroll
+    for (int j = 0; j < kUniqueItems; ++j) {
+        const int64_t i = first + j;
+        word[j] = i < n_valid ? __ldcs(keys + i) : 0ull;
+        const u64 key = word[j] >> val_bits;
+        if (i < n_valid && (i == 0 || key != prev)) mask |= 1u << j;
+        prev = key;
+    }
+    return mask;
+}
+
+// sum of one value per thread over the block, and the exclusive prefix of this thread's value
+__device__ __forceinline__ int32_t block_prefix_256(int32_t v, int32_t* total, int32_t* smem /*[8]*/)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    int32_t off = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+        const int32_t t = smem[w];
+        if (w < warp) off += t;
+        all += t;
+    }
+    *total = all;
+    return off + inc - v;
 }
 
 __global__ void __launch_bounds__(kThreads)
-compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const int32_t* __restrict__ flag,
-               const int32_t* __restrict__ pos, int64_t m, int val_bits, u64* __restrict__ keys_out,
-               int32_t* __restrict__ perm, BuildCounts* __restrict__ counts)
+unique_tile_counts(const u64* __restrict__ keys, int val_bits, const BuildCounts* __restrict__ counts,
+                   int32_t* __restrict__ tile_count)
 {
-    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (i >= m) return;
-    if (flag[i]) {
-        keys_out[pos[i]] = keys[i];
-        perm[pos[i]] = vals ? vals[i] : (int32_t)(keys[i] & ((1ull << val_bits) - 1ull)) - 1;
+    __shared__ int32_t smem[kThreads / 32];
+    u64 word[kUniqueItems];
+    const int64_t first = (int64_t)blockIdx.x * kUniqueTile + (int64_t)threadIdx.x * kUniqueItems;
+    const int32_t mine = __popc(first_of_run_mask(keys, first, counts->n_valid, val_bits, word));
+    int32_t total;
+    block_prefix_256(mine, &total, smem);
+    if (threadIdx.x == 0) tile_count[blockIdx.x] = total;
+}
+
+// tile_first[t] = kept candidates in earlier tiles; the kept ones move to keys_out / perm in order
+__global__ void __launch_bounds__(kThreads)
+compact_unique(const u64* __restrict__ keys, const int32_t* __restrict__ vals, const int32_t* __restrict__ tile_first,
+               int64_t m, int val_bits, u64* __restrict__ keys_out, int32_t* __restrict__ perm,
+               BuildCounts* __restrict__ counts)
+{
+    __shared__ int32_t smem[kThreads / 32];
+    __shared__ u64 kept_key[kUniqueTile];
+    __shared__ int32_t kept_val[kUniqueTile];
+    u64 word[kUniqueItems];
+    const int64_t first = (int64_t)blockIdx.x * kUniqueTile + (int64_t)threadIdx.x * kUniqueItems;
+    const uint32_t mask = first_of_run_mask(keys, first, counts->n_valid, val_bits, word);
+    int32_t total;
+    int32_t pos = block_prefix_256(__popc(mask), &total, smem);
+    // the kept candidates of the tile are gathered in shared memory so that they leave as one contiguous piece
+#pragma unroll
+    for (int j = 0; j < kUniqueItems; ++j) {
+        if (mask >> j & 1u) {
+            kept_key[pos] = word[j];
+            kept_val[pos] = vals ? vals[first + j] : (int32_t)(word[j] & ((1ull << val_bits) - 1ull)) - 1;
+            ++pos;
+        }
     }
-    if (i == m - 1) counts->nnz = pos[i] + flag[i];
+    __syncthreads();
+    const int32_t out0 = tile_first[blockIdx.x];
+    for (int i = threadIdx.x; i < total; i += kThreads) {
+        keys_out[out0 + i] = kept_key[i];
+        perm[out0 + i] = kept_val[i];
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) counts->nnz = tile_first[blockIdx.x] + total;
 }
 
 // row_ptr[v] = number of kept keys with dst < v (binary search in the sorted keys).  Without
@@ -553,14 +620,14 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
             int32_t* tv = vals; vals = vals_alt; vals_alt = tv;
         }
         if (dedup) {
-            GNNFD_LAUNCH("flag_first_of_run", s, flag_first_of_run, blocks_for(m, kThreads), kThreads, 0, keys, m, vb,
-                         P.counts, S.flags);
-            int32_t* pos = vals_alt;   // free after the last pass
-            rc = exclusive_scan_i32(S.flags, pos, (size_t)m, S.scan_temp, s);
+            const unsigned unique_tiles = blocks_for(m, kUniqueTile);
+            int32_t* tile_first = S.flags;
+            GNNFD_LAUNCH("unique_tile_counts", s, unique_tile_counts, unique_tiles, kThreads, 0, keys, vb, P.counts, tile_first);
+            rc = exclusive_scan_i32(tile_first, tile_first, (size_t)unique_tiles, S.scan_temp, s);
             if (rc) return rc;
-            GNNFD_LAUNCH("compact_unique", s, compact_unique, blocks_for(m, kThreads), kThreads, 0, keys,
-                         packed ? (const int32_t*)nullptr : (const int32_t*)vals, S.flags, pos, m, vb, keys_alt, P.perm,
-                         P.counts);
+            GNNFD_LAUNCH("compact_unique", s, compact_unique, unique_tiles, kThreads, 0, keys,
+                         packed ? (const int32_t*)nullptr : (const int32_t*)vals, (const int32_t*)tile_first, m, vb, keys_alt,
+                         P.perm, P.counts);
             u64* tk = keys; keys = keys_alt; keys_alt = tk;
         }
     }
