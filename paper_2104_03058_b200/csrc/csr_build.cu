@@ -15,10 +15,17 @@ using u64 = unsigned long long;
 constexpr int kThreads = 256;
 constexpr int kMaxDigitBits = 9;
 constexpr int kRadix = 1 << kMaxDigitBits;           // histogram bins (a pass may use fewer)
-constexpr int kSortItems = 16;                       // keys per thread
-constexpr int kSortTile = kThreads * kSortItems;     // keys per block
-constexpr int kSortWarps = kThreads / 32;
+constexpr int kSortTile = 4096;                      // keys per block of a sort pass
+#ifndef GNNFD_SCATTER_THREADS
+#define GNNFD_SCATTER_THREADS 256
+#endif
+constexpr int kHistItems = kSortTile / kThreads;     // keys per thread of the histogram kernel
+constexpr int kScatterThreads = GNNFD_SCATTER_THREADS;
+constexpr int kSortItems = kSortTile / kScatterThreads;   // keys per thread of the scatter kernel
+constexpr int kSortWarps = kScatterThreads / 32;
 constexpr int kWarpItems = 32 * kSortItems;
+constexpr int kOwnDigits = kRadix / kScatterThreads; // digit values a scatter thread looks after
+static_assert(kRadix % kScatterThreads == 0 && kOwnDigits >= 1, "a scatter block must cover the digit values evenly");
 
 static inline unsigned blocks_for(size_t count, int per_block)
 {
@@ -86,17 +93,17 @@ radix_histogram(const u64* __restrict__ keys, int64_t m, int shift, int mask, in
     if (base + kSortTile <= m) {
         // full tile: 16-byte loads, all of them issued before the first shared-memory atomic
         const ulonglong2* k2 = reinterpret_cast<const ulonglong2*>(keys + base);
-        ulonglong2 v[kSortItems / 2];
+        ulonglong2 v[kHistItems / 2];
 #pragma unroll
-        for (int i = 0; i < kSortItems / 2; ++i) v[i] = __ldcs(k2 + i * kThreads + threadIdx.x);
+        for (int i = 0; i < kHistItems / 2; ++i) v[i] = __ldcs(k2 + i * kThreads + threadIdx.x);
 #pragma unroll
-        for (int i = 0; i < kSortItems / 2; ++i) {
+        for (int i = 0; i < kHistItems / 2; ++i) {
             atomicAdd(&h[(int)(v[i].x >> shift) & mask], 1);
             atomicAdd(&h[(int)(v[i].y >> shift) & mask], 1);
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < kSortItems; ++i) {
+        for (int i = 0; i < kHistItems; ++i) {
             const int64_t idx = base + i * kThreads + threadIdx.x;
             if (idx < m) atomicAdd(&h[(int)(keys[idx] >> shift) & mask], 1);
         }
@@ -115,8 +122,8 @@ struct ScatterSmem {
     int32_t vals[kSortTile];        // last: not allocated when the values travel inside the keys
 };
 
-// exclusive scan of one value per thread over the block; *total receives the block sum
-__device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int32_t* smem)
+// exclusive scan of one value per thread over a scatter block; *total receives the block sum
+__device__ __forceinline__ int32_t block_scan(int32_t v, int32_t* total, int32_t* smem)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int32_t inc = v;
@@ -139,8 +146,8 @@ __device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int
     return off + inc - v;
 }
 
-// Stable scatter of one tile.  A warp owns 512 consecutive keys and walks them 32 at a time: keys with
-// equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp running
+// Stable scatter of one tile.  A warp owns kWarpItems consecutive keys and walks them 32 at a time: keys
+// with equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp running
 // count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
 // digit in shared memory and written out run by run, so that consecutive threads store to
 // consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
@@ -148,7 +155,7 @@ __device__ __forceinline__ int32_t block_scan_256(int32_t v, int32_t* total, int
 #define GNNFD_SCATTER_MIN_BLOCKS 3
 #endif
 template <bool HAS_VALS>
-__global__ void __launch_bounds__(kThreads, GNNFD_SCATTER_MIN_BLOCKS)
+__global__ void __launch_bounds__(kScatterThreads, GNNFD_SCATTER_MIN_BLOCKS)
 radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_in, u64* __restrict__ keys_out,
               int32_t* __restrict__ vals_out, int64_t m, int shift, int mask, int64_t n_tiles,
               const int32_t* __restrict__ tile_offset)
@@ -156,11 +163,7 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
     extern __shared__ __align__(16) unsigned char smem_raw[];
     ScatterSmem& sm = *reinterpret_cast<ScatterSmem*>(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int w = 0; w < kSortWarps; ++w) {
-        sm.warp_count[w][threadIdx.x] = 0;
-        sm.warp_count[w][threadIdx.x + kThreads] = 0;
-    }
+    for (int i = threadIdx.x; i < kSortWarps * kRadix; i += kScatterThreads) (&sm.warp_count[0][0])[i] = 0;
     __syncthreads();
 
     const int64_t tile_base = (int64_t)blockIdx.x * kSortTile;
@@ -187,11 +190,11 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
     }
     __syncthreads();
     {
-        // per-warp counts -> exclusive prefix over warps; thread t owns digits t and t + 256
-        int32_t tot[2];
+        // per-warp counts -> exclusive prefix over warps; thread t owns digit values t, t + blockDim, ...
+        int32_t carry = 0;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int d = threadIdx.x + half * kThreads;
+        for (int q = 0; q < kOwnDigits; ++q) {
+            const int d = threadIdx.x + q * kScatterThreads;
             int32_t run = 0;
 #pragma unroll
             for (int w = 0; w < kSortWarps; ++w) {
@@ -199,16 +202,12 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
                 sm.warp_count[w][d] = run;
                 run += c;
             }
-            tot[half] = run;
+            int32_t total;
+            const int32_t base = block_scan(run, &total, sm.scan) + carry;
+            carry += total;
+            sm.digit_base[d] = base;
+            sm.to_global[d] = tile_offset[(int64_t)d * n_tiles + blockIdx.x] - base;
         }
-        int32_t low_total, high_total;
-        const int32_t base0 = block_scan_256(tot[0], &low_total, sm.scan);
-        const int32_t base1 = block_scan_256(tot[1], &high_total, sm.scan) + low_total;
-        sm.digit_base[threadIdx.x] = base0;
-        sm.digit_base[threadIdx.x + kThreads] = base1;
-        sm.to_global[threadIdx.x] = tile_offset[(int64_t)threadIdx.x * n_tiles + blockIdx.x] - base0;
-        sm.to_global[threadIdx.x + kThreads] =
-            tile_offset[(int64_t)(threadIdx.x + kThreads) * n_tiles + blockIdx.x] - base1;
     }
     __syncthreads();
 #pragma unroll
@@ -222,7 +221,7 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
     }
     __syncthreads();
     const int count = (int)min((int64_t)kSortTile, m - tile_base);
-    for (int i = threadIdx.x; i < count; i += kThreads) {
+    for (int i = threadIdx.x; i < count; i += kScatterThreads) {
         const u64 k = sm.keys[i];
         const int64_t pos = (int64_t)sm.to_global[(int)(k >> shift) & mask] + i;
         keys_out[pos] = k;
@@ -611,10 +610,10 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
             rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.n_tiles, S.scan_temp, s);
             if (rc) return rc;
             if (packed)
-                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<false>, (unsigned)L.n_tiles, kThreads, scatter_smem, keys,
+                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<false>, (unsigned)L.n_tiles, kScatterThreads, scatter_smem, keys,
                              (const int32_t*)nullptr, keys_alt, (int32_t*)nullptr, m, shift, mask, L.n_tiles, S.hist);
             else
-                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.n_tiles, kThreads, scatter_smem, keys,
+                GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.n_tiles, kScatterThreads, scatter_smem, keys,
                              (const int32_t*)vals, keys_alt, vals_alt, m, shift, mask, L.n_tiles, S.hist);
             u64* tk = keys; keys = keys_alt; keys_alt = tk;
             int32_t* tv = vals; vals = vals_alt; vals_alt = tv;
@@ -646,7 +645,7 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
                      L.row_tiles, S.hist);
         rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.row_tiles, S.scan_temp, s);
         if (rc) return rc;
-        GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.row_tiles, kThreads, sizeof(ScatterSmem), keys_alt,
+        GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.row_tiles, kScatterThreads, sizeof(ScatterSmem), keys_alt,
                      vals_alt, reinterpret_cast<u64*>(S.flags), P.row_order, n, 32, kRadix - 1, L.row_tiles, S.hist);
     }
     // the flag buffer is free again: per-hub-row segment counts

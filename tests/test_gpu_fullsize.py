@@ -119,3 +119,23 @@ def test_config4_graph_edge_softmax_sampled_rows(big):
     row_of_slot = torch.repeat_interleave(torch.arange(w.n, device="cuda"), torch.from_numpy(deg).cuda().long())
     sums.index_add_(0, row_of_slot, alpha.double())
     assert float((sums - 1.0).abs().max()) <= 1e-5
+
+
+def test_config4_features_combined_to_64_columns_sampled_rows(big):
+    """The dense transform ahead of aggregation at the bench's size ([232,965, 602] in rows of 608 times a
+    [602, 64] matrix): sampled rows, the last partial row tile among them, against the oracle's tf32
+    reading (summation order only) and the exact product (the tf32 bound)."""
+    g, w, _, _ = big
+    f_out = 64
+    w_t = gg.features_f32(f_out, w.ld, dist="normal", p0=0.0, p1=0.05, seed=3, stream=8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    z = g.combine(torch.from_numpy(w.x).cuda()[:, :w.f], torch.from_numpy(w_t).cuda()[:, :w.f], status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rng = np.random.default_rng(7)
+    rows = np.unique(np.concatenate([rng.choice(w.n, 2000, replace=False), np.arange(w.n - 130, w.n), np.arange(130)]))
+    got = z[torch.from_numpy(rows).cuda()].cpu().numpy().astype(np.float64)
+    exact, scale = orc.combine(w.x[rows][:, :w.f], w_t[:, :w.f])
+    cut, _ = orc.combine(w.x[rows][:, :w.f], w_t[:, :w.f], tf32=True)
+    assert (np.abs(got - cut) <= 1e-5 * scale + 1e-6).all()
+    assert (np.abs(got - exact) <= 2.0 ** -9 * scale + 1e-6).all()
