@@ -395,6 +395,13 @@ def run_ours(args):
         combine_ms = a0.elapsed_time(a1) / 20
         del z, w_t
 
+    # what L2 delivers for random row reads of one chunk's slice with nothing else going on: the measured
+    # ceiling beside the L2 peak that ncu derives
+    l2_measured = None
+    slice_rows = min(w.n, out.numel() * 4 // 256)
+    if slice_rows * 256 <= 0.6 * l2_bytes:
+        l2_measured = g.measure_random_row_reads(out, slice_rows, 256)
+
     ms, total_units = sharding.reduce_job_timing(ms, float(units_per_step), device=device)
     ms_e2e, _ = sharding.reduce_job_timing(ms_e2e, 0.0, device=device)
 
@@ -428,7 +435,9 @@ def run_ours(args):
                             "achieved": achieved, "peak": L2_PEAK_BYTES_PER_CLK * (clocks["sm_max_mhz"] or 1965.0) / 1e3,
                             "unit": "GB/s",
                             "frac": achieved / (L2_PEAK_BYTES_PER_CLK * (clocks["sm_max_mhz"] or 1965.0) / 1e3)
-                            if achieved else None},
+                            if achieved else None,
+                            "measured_random_row_read_GBs": l2_measured,
+                            "frac_of_measured": achieved / l2_measured if achieved and l2_measured else None},
             "e2e": {"value": total_units * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,

@@ -252,6 +252,15 @@ int64_t gnnfd_launch_count(void);
 int gnnfd_kernel_timing_enable(int on);
 int gnnfd_kernel_timing_read(const char** names, double* ms, int64_t* launches, int capacity);
 
+/* Measurement aid for the roofline of the gather kernels (which are bound by L2-to-SM bandwidth when a
+ * chunk's slice is resident, not by HBM): reads 256-byte rows, drawn uniformly at random by an integer
+ * hash from `rows` rows that lie pitch_bytes apart in d_buf, with nothing else going on, and reports
+ * the rate of the best of three timed launches in *gb_per_s.  d_buf is only read (any contents), must be
+ * 16-byte aligned and hold rows * pitch_bytes bytes; pitch_bytes >= 256 and a multiple of 16.
+ * Synchronises the stream. */
+int gnnfd_measure_random_row_reads(const void* d_buf, size_t buf_bytes, int64_t rows, int64_t pitch_bytes,
+                                   void* stream, double* gb_per_s);
+
 #ifdef __cplusplus
 }
 #endif

@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_edge_softmax_workspace_bytes.argtypes = [vp, i32, pp(sz)]
         L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp, sz, vp]
         L.gnnfd_combine.argtypes = [i64, vp, i64, i32, i32, vp, i64, i32, vp, i64, i32, vp, vp]
+        L.gnnfd_measure_random_row_reads.argtypes = [vp, sz, i64, i64, vp, pp(ctypes.c_double)]
         L.gnnfd_status_string.argtypes = [ctypes.c_int]
         L.gnnfd_status_string.restype = ctypes.c_char_p
         L.gnnfd_last_cuda_error.restype = ctypes.c_int
@@ -359,6 +360,15 @@ def combine(x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, out: to
     _check(lib().gnnfd_combine(x.shape[0], xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, op, ldo, _dtype_code(out), sp,
                                _stream_ptr(stream)), "gnnfd_combine")
     return out
+
+
+def measure_random_row_reads(buf: torch.Tensor, rows: int, pitch_bytes: int = 256, stream=None) -> float:
+    """gnnfd_measure_random_row_reads: GB/s at which random 256-byte rows of a resident set reach the SMs."""
+    out = ctypes.c_double()
+    _check(lib().gnnfd_measure_random_row_reads(ctypes.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size(), rows,
+                                                pitch_bytes, _stream_ptr(stream), ctypes.byref(out)),
+           "gnnfd_measure_random_row_reads")
+    return out.value
 
 
 def launch_count() -> int:

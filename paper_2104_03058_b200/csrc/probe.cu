@@ -1,0 +1,86 @@
+// Measurement aid: how fast this GPU serves random row reads out of a resident working set.  The
+// gather kernels read rows of a chunk's slice in an order set by the graph; when the slice fits L2
+// their ceiling is what L2 delivers to the SMs for such reads, which no copy benchmark measures.
+// This kernel does only that: lanes in groups of eight read 256-byte rows (two 16-byte loads per
+// lane, eight rows in flight per group) whose numbers come from an integer hash, with no index stream,
+// no arithmetic worth the name and no output.
+#include "common.cuh"
+
+namespace gnnfd {
+
+constexpr int kProbeThreads = 256;
+constexpr int kProbeLanes = 8;          // lanes per row
+constexpr int kProbeRowsInFlight = 8;
+constexpr int kProbeRowBytes = kProbeLanes * 2 * 16;
+
+__device__ __forceinline__ uint32_t probe_hash(uint32_t x)
+{
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
+__global__ void __launch_bounds__(kProbeThreads, 3)
+random_row_reads(const float4* __restrict__ buf, uint32_t rows, uint32_t pitch_v4, int rounds, float* __restrict__ sink)
+{
+    const int c = threadIdx.x % kProbeLanes;
+    const uint32_t group = (blockIdx.x * (uint32_t)kProbeThreads + threadIdx.x) / kProbeLanes;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t state = probe_hash(group * 2654435761u + 12345u);
+    for (int it = 0; it < rounds; ++it) {
+        float4 v[kProbeRowsInFlight][2];
+#pragma unroll
+        for (int i = 0; i < kProbeRowsInFlight; ++i) {
+            state = state * 1664525u + 1013904223u;
+            const uint32_t row = (uint32_t)(((uint64_t)probe_hash(state) * rows) >> 32);      // < rows
+            const float4* p = buf + (size_t)row * pitch_v4 + c;
+            v[i][0] = __ldg(p);
+            v[i][1] = __ldg(p + kProbeLanes);
+        }
+#pragma unroll
+        for (int i = 0; i < kProbeRowsInFlight; ++i) {
+            acc.x += v[i][0].x + v[i][1].x; acc.y += v[i][0].y + v[i][1].y;
+            acc.z += v[i][0].z + v[i][1].z; acc.w += v[i][0].w + v[i][1].w;
+        }
+    }
+    if (sink && acc.x + acc.y + acc.z + acc.w == 1.2345e-30f) sink[0] = acc.x;      // keeps the loads alive
+}
+
+}  // namespace gnnfd
+
+extern "C" int gnnfd_measure_random_row_reads(const void* d_buf, size_t buf_bytes, int64_t rows, int64_t pitch_bytes,
+                                              void* stream, double* gb_per_s)
+{
+    using namespace gnnfd;
+    if (!d_buf || !gb_per_s || rows <= 0 || rows > 0x7fffffffll || pitch_bytes < kProbeRowBytes || pitch_bytes % 16 != 0 ||
+        ((uintptr_t)d_buf & 15u))
+        return GNNFD_INVALID_ARG;
+    if ((size_t)rows * (size_t)pitch_bytes > buf_bytes) return GNNFD_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int sms = 0, dev = 0;
+    GNNFD_CUDA_CHECK(cudaGetDevice(&dev));
+    GNNFD_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const unsigned grid = (unsigned)(sms * 3);
+    const int rounds = 2000;
+    cudaEvent_t e0, e1;
+    GNNFD_CUDA_CHECK(cudaEventCreate(&e0));
+    GNNFD_CUDA_CHECK(cudaEventCreate(&e1));
+    float best = 0.f;
+    int rc = GNNFD_OK;
+    for (int rep = 0; rep < 4 && rc == GNNFD_OK; ++rep) {            // the first launch warms the working set
+        cudaEventRecord(e0, s);
+        GNNFD_LAUNCH("random_row_reads", s, random_row_reads, grid, kProbeThreads, 0, static_cast<const float4*>(d_buf),
+                     (uint32_t)rows, (uint32_t)(pitch_bytes / 16), rounds, (float*)nullptr);
+        cudaEventRecord(e1, s);
+        float ms = 0.f;
+        cudaError_t err = cudaEventSynchronize(e1);
+        if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
+        if (err != cudaSuccess) { set_cuda_error(err); rc = GNNFD_CUDA_ERROR; break; }
+        if (rep > 0 && (best == 0.f || ms < best)) best = ms;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc != GNNFD_OK) return rc;
+    const double bytes = (double)grid * kProbeThreads / kProbeLanes * rounds * kProbeRowsInFlight * (double)kProbeRowBytes;
+    *gb_per_s = bytes / (best * 1e-3) / 1e9;
+    return GNNFD_OK;
+}

@@ -451,3 +451,16 @@ def test_csr_sort_boundaries(g, n, e, flags):
     assert torch.equal(csr.col_idx.cpu(), torch.from_numpy(col))
     assert torch.equal(csr.perm.cpu(), torch.from_numpy(perm))
     assert sum(csr.bin_count) == n
+
+
+def test_random_row_read_measurement(g):
+    buf = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
+    rate = g.measure_random_row_reads(buf, rows=(8 << 20) // 256, pitch_bytes=256)
+    assert rate > 100.0                                   # GB/s; any B200 is far above this
+    strided = g.measure_random_row_reads(buf, rows=(8 << 20) // 512, pitch_bytes=512)
+    assert strided > 100.0
+    with pytest.raises(g.GnnfdError) as err:              # more rows than the buffer holds
+        g.measure_random_row_reads(buf, rows=(8 << 20) // 256 + 1, pitch_bytes=256)
+    assert err.value.status == g.WORKSPACE_TOO_SMALL
+    with pytest.raises(g.GnnfdError):
+        g.measure_random_row_reads(buf, rows=16, pitch_bytes=128)
