@@ -506,8 +506,9 @@ struct ScratchPtrs {
 
 static size_t flag_ints(int64_t n, const BuildLayout& L)
 {
-    // dedup flags (m), a 64-bit dump for the row sort's keys (2 ints per row), hub segment counts
-    size_t a = (size_t)L.m, b = 2 * (size_t)n + 2, c = (size_t)L.hub_cap + 1;
+    // one count per tile of the duplicate removal, a 64-bit dump for the row sort's keys (2 ints per row),
+    // hub segment counts
+    size_t a = (size_t)L.m / kUniqueTile + 2, b = 2 * (size_t)n + 2, c = (size_t)L.hub_cap + 1;
     size_t r = a > b ? a : b;
     return (r > c ? r : c) + 1;
 }
@@ -517,8 +518,10 @@ static void carve_scratch(Carver& c, int64_t n, const BuildLayout& L, ScratchPtr
     const size_t cap = (size_t)(L.m > n ? L.m : n);      // the row sort reuses the edge sort's buffers
     p->keys_a = c.take<u64>(cap);
     p->keys_b = c.take<u64>(cap);
-    p->vals_a = c.take<int32_t>(cap);
-    p->vals_b = c.take<int32_t>(cap);
+    // when the values travel inside the key words only the row sort needs value buffers
+    const size_t val_cap = L.val_bits > 0 ? (size_t)n : cap;
+    p->vals_a = c.take<int32_t>(val_cap);
+    p->vals_b = c.take<int32_t>(val_cap);
     const size_t hist_ints = (size_t)kRadix * (size_t)(L.n_tiles > L.row_tiles ? L.n_tiles : L.row_tiles);
     p->hist = c.take<int32_t>(hist_ints);
     const size_t fl = flag_ints(n, L);
