@@ -442,6 +442,16 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,
             "clocks": clocks,
+            # device memory of one step (the paper's second axis, Fig. 6): the build scratch may be freed after the build
+            "device_memory_bytes": {
+                "edge_list": d_src.numel() * d_src.element_size() * 2,
+                "features": d_x.numel() * d_x.element_size(), "output": out.numel() * 4,
+                "csr_persistent": pb, "build_scratch": sb,
+                "aggregation_scratch": state["agg_scratch"].numel() if state["agg_scratch"] is not None else 0,
+                "total_during_build": d_src.numel() * d_src.element_size() * 2 + d_x.numel() * d_x.element_size()
+                                      + out.numel() * 4 + pb + sb,
+                "total_after_build": d_x.numel() * d_x.element_size() + out.numel() * 4 + pb
+                                     + (state["agg_scratch"].numel() if state["agg_scratch"] is not None else 0)},
             "kernels": {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps,
                             "share": v[0] / total_kernel_ms if total_kernel_ms else None}
                         for k, v in sorted(kernels.items(), key=lambda kv: -kv[1][0])},
