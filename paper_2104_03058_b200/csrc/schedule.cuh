@@ -10,7 +10,6 @@ namespace gnnfd {
 #define GNNFD_GATHER_BLOCK 256
 #endif
 constexpr int kBlock = GNNFD_GATHER_BLOCK;      // threads per block of the gather kernels
-constexpr int kUnroll = 8;       // loads kept in flight per lane
 constexpr int kMaxRanges = 5;
 
 struct Range {
