@@ -139,3 +139,32 @@ def test_config4_features_combined_to_64_columns_sampled_rows(big):
     cut, _ = orc.combine(w.x[rows][:, :w.f], w_t[:, :w.f], tf32=True)
     assert (np.abs(got - cut) <= 1e-5 * scale + 1e-6).all()
     assert (np.abs(got - exact) <= 2.0 ** -9 * scale + 1e-6).all()
+
+
+def test_config5_full_size_csr_and_bf16_aggregation():
+    """Config 5 at its full size (RMAT scale 21, 60M edges, symmetrised + deduplicated + self-loops, bf16
+    features of width 64): the CSR bit for bit, the kept-entry count against a direct count of distinct
+    off-diagonal pairs, and the aggregation on sampled rows of every degree class."""
+    import paper_2104_03058_b200 as g
+    w = gg.config5(f=64)
+    row_ptr, col, perm = orc.build_csr(w.n, w.src, w.dst, w.flags)
+    csr = g.build_csr(w.n, torch.from_numpy(w.src).cuda(), torch.from_numpy(w.dst).cuda(), w.flags)
+    assert csr.nnz == len(col)
+    assert torch.equal(csr.row_ptr.cpu(), torch.from_numpy(row_ptr))
+    assert torch.equal(csr.col_idx.cpu(), torch.from_numpy(col))
+    assert torch.equal(csr.perm.cpu(), torch.from_numpy(perm))
+    # distinct undirected pairs, both directions, plus one loop per vertex
+    a, b = w.src.astype(np.int64), w.dst.astype(np.int64)
+    off = a != b
+    pairs = np.unique(np.minimum(a[off], b[off]) * w.n + np.maximum(a[off], b[off]))
+    assert csr.nnz == 2 * len(pairs) + w.n
+    deg = np.diff(row_ptr)
+    rng = np.random.default_rng(8)
+    rows = np.unique(np.concatenate([rng.choice(w.n, 256, replace=False), np.argsort(deg)[-8:], np.argsort(deg)[:8]]))
+    rows = rows.astype(np.int64)
+    want, scale = orc.aggregate("gcn", row_ptr, col, w.x, w.f, rows=rows, threads=orc.max_threads())
+    xd = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16)
+    sel = torch.from_numpy(rows).cuda()
+    for width in (64, 8):
+        got = g.aggregate_gcn(csr, xd, f=w.f, chunk_width=width)[sel].cpu().numpy()
+        assert (np.abs(got - want) <= 1e-2 * np.abs(want) + 1e-5 * scale + 1e-6).all(), "width %d" % width
