@@ -30,7 +30,11 @@ namespace gnnfd {
 #ifndef GNNFD_SOFTMAX_MIN_BLOCKS
 #define GNNFD_SOFTMAX_MIN_BLOCKS 4
 #endif
-constexpr int kSlotsInFlight = GNNFD_SOFTMAX_IN_FLIGHT;      // slots a lane has in flight
+// slots a lane has in flight when it holds HB heads of a slot: GNNFD_SOFTMAX_IN_FLIGHT 16-byte loads' worth, at most 16
+template <int HB> constexpr int slots_in_flight()
+{
+    return GNNFD_SOFTMAX_IN_FLIGHT * 4 / HB > 16 ? 16 : GNNFD_SOFTMAX_IN_FLIGHT * 4 / HB < 2 ? 2 : GNNFD_SOFTMAX_IN_FLIGHT * 4 / HB;
+}
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct SoftmaxArgs {
@@ -103,21 +107,21 @@ struct Leaky {
 };
 
 // column indices of slots k, k + SP, ... of one row (-1 past the end of the row)
-template <int SP>
-__device__ __forceinline__ void load_cols(const SoftmaxArgs& a, int32_t k, int32_t e, int32_t (&u)[kSlotsInFlight])
+template <int SP, int NF>
+__device__ __forceinline__ void load_cols(const SoftmaxArgs& a, int32_t k, int32_t e, int32_t (&u)[NF])
 {
 #pragma unroll
-    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = k + i * SP < e ? __ldg(a.col_idx + k + i * SP) : -1;
+    for (int i = 0; i < NF; ++i) u[i] = k + i * SP < e ? __ldg(a.col_idx + k + i * SP) : -1;
 }
 
 // base-2 logits of the slots whose column indices are u[].  FULL: all of them exist; otherwise the
 // missing ones (u < 0) get -inf.
-template <int HB, bool FULL>
+template <int HB, bool FULL, int NF>
 __device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const Leaky& leaky, const float* ssrc, const float (&sd)[HB],
-                                            const int32_t (&u)[kSlotsInFlight], float (&t)[kSlotsInFlight][HB])
+                                            const int32_t (&u)[NF], float (&t)[NF][HB])
 {
 #pragma unroll
-    for (int i = 0; i < kSlotsInFlight; ++i) {
+    for (int i = 0; i < NF; ++i) {
         if (FULL || u[i] >= 0) {
             load_heads<HB>(ssrc + (int64_t)u[i] * a.heads, t[i]);
         } else {
@@ -126,7 +130,7 @@ __device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const Leaky& l
         }
     }
 #pragma unroll
-    for (int i = 0; i < kSlotsInFlight; ++i)
+    for (int i = 0; i < NF; ++i)
 #pragma unroll
         for (int h = 0; h < HB; ++h) {
             const float y = leaky(t[i][h] + sd[h]);
@@ -135,17 +139,17 @@ __device__ __forceinline__ void load_logits(const SoftmaxArgs& a, const Leaky& l
 }
 
 // running (max, sum) of one head over a batch of logits
-template <int HB>
-__device__ __forceinline__ void online_update(const float (&t)[kSlotsInFlight][HB], float (&m)[HB], float (&l)[HB])
+template <int HB, int NF>
+__device__ __forceinline__ void online_update(const float (&t)[NF][HB], float (&m)[HB], float (&l)[HB])
 {
 #pragma unroll
     for (int h = 0; h < HB; ++h) {
         float mx = m[h];                                               // t[0] is a real slot, so mx ends finite
 #pragma unroll
-        for (int i = 0; i < kSlotsInFlight; ++i) mx = fmaxf(mx, t[i][h]);
+        for (int i = 0; i < NF; ++i) mx = fmaxf(mx, t[i][h]);
         float sum = 0.f;
 #pragma unroll
-        for (int i = 0; i < kSlotsInFlight; ++i) sum += ex2(t[i][h] - mx);                  // 2^-inf = 0
+        for (int i = 0; i < NF; ++i) sum += ex2(t[i][h] - mx);                  // 2^-inf = 0
         l[h] = l[h] * ex2(m[h] - mx) + sum;
         m[h] = mx;
     }
@@ -158,6 +162,7 @@ template <int HB, int LPS, int SP, int MODE>
 __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range& rg, int block_in_range)
 {
     constexpr int S = LPS * SP;
+    constexpr int NF = slots_in_flight<HB>();
     constexpr unsigned kFull = 0xffffffffu;
     const int tid = threadIdx.x;
     const int slot = block_in_range * (kBlock / S) + tid / S;
@@ -178,7 +183,7 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
         }
     }
     // every row of the warp fits one batch: the write pass reuses the logits of the first pass
-    const bool fits = MODE == kModeRows && __all_sync(kFull, e - b <= SP * kSlotsInFlight);
+    const bool fits = MODE == kModeRows && __all_sync(kFull, e - b <= SP * NF);
     const Leaky leaky(a.slope);
 
     for (int hh = 0; hh < a.heads; hh += LPS * HB) {
@@ -190,27 +195,27 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
         if (active && head_ok) load_heads<HB>(a.s_dst + (int64_t)row * a.heads + h0, sd);
         const float* ssrc = a.s_src + h0;
         float m[HB], inv[HB];
-        float t[kSlotsInFlight][HB];
+        float t[NF][HB];
 
         if (MODE != kModeHubWrite) {
             float l[HB];
 #pragma unroll
             for (int h = 0; h < HB; ++h) { m[h] = -CUDART_INF_F; l[h] = 0.f; }
             if (head_ok) {
-                int32_t u[kSlotsInFlight], un[kSlotsInFlight];
-                load_cols<SP>(a, b + sp, e, u);
-                for (int32_t kb = b; kb < e; kb += SP * kSlotsInFlight) {
+                int32_t u[NF], un[NF];
+                load_cols<SP, NF>(a, b + sp, e, u);
+                for (int32_t kb = b; kb < e; kb += SP * NF) {
                     // the next batch's indices are on their way while this batch is gathered and reduced
-                    load_cols<SP>(a, kb + SP * kSlotsInFlight + sp, e, un);
-                    if (kb + SP * kSlotsInFlight <= e) {               // the same for all lanes of the row
-                        load_logits<HB, true>(a, leaky, ssrc, sd, u, t);
-                        online_update<HB>(t, m, l);
+                    load_cols<SP, NF>(a, kb + SP * NF + sp, e, un);
+                    if (kb + SP * NF <= e) {               // the same for all lanes of the row
+                        load_logits<HB, true, NF>(a, leaky, ssrc, sd, u, t);
+                        online_update<HB, NF>(t, m, l);
                     } else if (u[0] >= 0) {
-                        load_logits<HB, false>(a, leaky, ssrc, sd, u, t);
-                        online_update<HB>(t, m, l);
+                        load_logits<HB, false, NF>(a, leaky, ssrc, sd, u, t);
+                        online_update<HB, NF>(t, m, l);
                     }
 #pragma unroll
-                    for (int i = 0; i < kSlotsInFlight; ++i) u[i] = un[i];
+                    for (int i = 0; i < NF; ++i) u[i] = un[i];
                 }
             }
             // butterfly over the SP lanes that hold the same heads; both partners evaluate the same commutative expression
@@ -246,7 +251,7 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
 
         if (fits) {
 #pragma unroll
-            for (int i = 0; i < kSlotsInFlight; ++i) {
+            for (int i = 0; i < NF; ++i) {
                 const int32_t k = b + sp + i * SP;
                 if (k < e) {
                     float w[HB];
@@ -256,24 +261,24 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
                 }
             }
         } else {
-            int32_t u[kSlotsInFlight], un[kSlotsInFlight];
-            load_cols<SP>(a, b + sp, e, u);
-            for (int32_t kb = b; kb < e; kb += SP * kSlotsInFlight) {
+            int32_t u[NF], un[NF];
+            load_cols<SP, NF>(a, b + sp, e, u);
+            for (int32_t kb = b; kb < e; kb += SP * NF) {
                 const int32_t k = kb + sp;
-                load_cols<SP>(a, k + SP * kSlotsInFlight, e, un);
-                if (kb + SP * kSlotsInFlight <= e) {
-                    load_logits<HB, true>(a, leaky, ssrc, sd, u, t);
+                load_cols<SP, NF>(a, k + SP * NF, e, un);
+                if (kb + SP * NF <= e) {
+                    load_logits<HB, true, NF>(a, leaky, ssrc, sd, u, t);
 #pragma unroll
-                    for (int i = 0; i < kSlotsInFlight; ++i) {
+                    for (int i = 0; i < NF; ++i) {
                         float w[HB];
 #pragma unroll
                         for (int h = 0; h < HB; ++h) w[h] = ex2(t[i][h] - m[h]) * inv[h];
                         store_heads<HB>(a.alpha + (int64_t)(k + i * SP) * a.heads + h0, w);
                     }
                 } else if (u[0] >= 0) {
-                    load_logits<HB, false>(a, leaky, ssrc, sd, u, t);
+                    load_logits<HB, false, NF>(a, leaky, ssrc, sd, u, t);
 #pragma unroll
-                    for (int i = 0; i < kSlotsInFlight; ++i) {
+                    for (int i = 0; i < NF; ++i) {
                         if (u[i] >= 0) {
                             float w[HB];
 #pragma unroll
@@ -283,7 +288,7 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
                     }
                 }
 #pragma unroll
-                for (int i = 0; i < kSlotsInFlight; ++i) u[i] = un[i];
+                for (int i = 0; i < NF; ++i) u[i] = un[i];
             }
         }
     }
