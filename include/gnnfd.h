@@ -6,8 +6,9 @@
  * Aggregate and Concat steps): the feature dimension is cut into chunks of
  * `chunk_width` columns, every chunk is aggregated over all vertices, and each
  * chunk's result is written into its own columns of the output.  The
- * Combination (dense) phase is the caller's; its output is this library's input
- * (Section III: combination is run ahead of aggregation).
+ * Combination (dense) phase comes first (Section III: combination is run ahead
+ * of aggregation); its output is the aggregation's input, whether the caller
+ * computed it or gnnfd_combine did.
  *
  * Conventions
  *   - Every pointer named d_* is DEVICE memory owned by the caller.  The library
@@ -51,7 +52,7 @@ typedef enum {
     GNNFD_BAD_INDEX = -2,           /* a vertex id outside [0, n) was found in the edge list */
     GNNFD_TOO_LARGE = -3,           /* n, e or the resulting nnz does not fit the int32 structure */
     GNNFD_WORKSPACE_TOO_SMALL = -4, /* a caller-provided buffer is smaller than the size query says */
-    GNNFD_UNSUPPORTED = -5,         /* unknown dtype / itype enum */
+    GNNFD_UNSUPPORTED = -5,         /* unknown dtype / itype enum; an operand layout gnnfd_combine cannot take */
     GNNFD_CUDA_ERROR = -6,          /* a CUDA runtime call failed; see gnnfd_last_cuda_error() */
     GNNFD_STATIC_SCRATCH_EXCEEDED = -7 /* the built-in workspace of a *_static entry point is too small for this call */
 } gnnfd_status_t;
