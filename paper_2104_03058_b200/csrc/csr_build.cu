@@ -40,43 +40,75 @@ static inline unsigned blocks_for(size_t count, int per_block)
 // destination n, above every valid key, so the sort moves them behind the kept ones.  When key and
 // value fit one 64-bit word together (vals == nullptr) the word is key << val_bits | (value + 1) and
 // every later kernel reads the key as word >> val_bits.
+constexpr int kKeyItems = 4;                          // candidates per thread of make_keys / entries per thread of finalize_entries
+
 template <typename IdT>
 __global__ void __launch_bounds__(kThreads)
 make_keys(const IdT* __restrict__ src, const IdT* __restrict__ dst, int64_t n, int64_t e, int64_t m, uint32_t flags,
           int src_bits, int val_bits, u64* __restrict__ keys, int32_t* __restrict__ vals,
           BuildCounts* __restrict__ counts)
 {
-    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * kKeyItems) + threadIdx.x;
     const u64 invalid = (u64)n << src_bits;
     const int64_t n_rev = (flags & GNNFD_CSR_SYMMETRIZE) ? e : 0;
-    bool keep = false, bad = false;
-    if (i < m) {
-        int64_t s, d;
-        int32_t val;
-        if (i < e) {
-            s = (int64_t)src[i]; d = (int64_t)dst[i]; val = (int32_t)i;
-            bad = s < 0 || s >= n || d < 0 || d >= n;
-            keep = !bad && !((flags & GNNFD_CSR_ADD_SELF_LOOPS) && s == d);
-        } else if (i < e + n_rev) {
-            s = (int64_t)dst[i - e]; d = (int64_t)src[i - e]; val = (int32_t)i;
-            keep = !(s < 0 || s >= n || d < 0 || d >= n) && s != d;
-        } else {
-            s = d = i - e - n_rev; val = -1;
-            keep = true;
-        }
-        const u64 key = keep ? (((u64)d << src_bits) | (u64)s) : invalid;
+    int kept = 0, bads = 0;
+    auto emit = [&](int64_t i, int64_t sv, int64_t dv, int32_t val, bool keep) {
+        const u64 key = keep ? (((u64)dv << src_bits) | (u64)sv) : invalid;
         if (vals) {
             __stcs(keys + i, key);
             __stcs(vals + i, val);
         } else {
             __stcs(keys + i, (key << val_bits) | (u64)(uint32_t)(val + 1));   // value travels in the low bits
         }
+        kept += keep ? 1 : 0;
+    };
+    if ((int64_t)(blockIdx.x + 1) * (kThreads * kKeyItems) <= e) {
+        // the block lies inside the plain input edges: all loads are issued before the first store
+        IdT sv[kKeyItems], dv[kKeyItems];
+#pragma unroll
+        for (int j = 0; j < kKeyItems; ++j) {
+            sv[j] = __ldcs(src + base + j * kThreads);
+            dv[j] = __ldcs(dst + base + j * kThreads);
+        }
+#pragma unroll
+        for (int j = 0; j < kKeyItems; ++j) {
+            const int64_t s64 = (int64_t)sv[j], d64 = (int64_t)dv[j];
+            const bool bad = s64 < 0 || s64 >= n || d64 < 0 || d64 >= n;
+            bads += bad ? 1 : 0;
+            emit(base + j * kThreads, s64, d64, (int32_t)(base + j * kThreads),
+                 !bad && !((flags & GNNFD_CSR_ADD_SELF_LOOPS) && s64 == d64));
+        }
+    } else {
+        for (int j = 0; j < kKeyItems; ++j) {
+            const int64_t i = base + j * kThreads;
+            if (i >= m) break;
+            if (i < e) {
+                const int64_t s64 = (int64_t)src[i], d64 = (int64_t)dst[i];
+                const bool bad = s64 < 0 || s64 >= n || d64 < 0 || d64 >= n;
+                bads += bad ? 1 : 0;
+                emit(i, s64, d64, (int32_t)i, !bad && !((flags & GNNFD_CSR_ADD_SELF_LOOPS) && s64 == d64));
+            } else if (i < e + n_rev) {
+                const int64_t s64 = (int64_t)dst[i - e], d64 = (int64_t)src[i - e];
+                emit(i, s64, d64, (int32_t)i, !(s64 < 0 || s64 >= n || d64 < 0 || d64 >= n) && s64 != d64);
+            } else {
+                emit(i, i - e - n_rev, i - e - n_rev, -1, true);
+            }
+        }
     }
-    const int kept = __syncthreads_count(keep);
-    const int bads = __syncthreads_count(bad);
+    // one atomic per block and counter: all blocks add to the same two words
+    __shared__ int warp_kept[kThreads / 32], warp_bads[kThreads / 32];
+    const int kept_warp = __reduce_add_sync(0xffffffffu, kept), bads_warp = __reduce_add_sync(0xffffffffu, bads);
+    if ((threadIdx.x & 31) == 0) {
+        warp_kept[threadIdx.x >> 5] = kept_warp;
+        warp_bads[threadIdx.x >> 5] = bads_warp;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
-        if (kept) atomicAdd(&counts->n_valid, kept);
-        if (bads) atomicAdd(&counts->bad_index, bads);
+        int kept_all = 0, bads_all = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) { kept_all += warp_kept[w]; bads_all += warp_bads[w]; }
+        if (kept_all) atomicAdd(&counts->n_valid, kept_all);
+        if (bads_all) atomicAdd(&counts->bad_index, bads_all);
     }
 }
 
@@ -390,15 +422,30 @@ finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals,
                  const BuildCounts* __restrict__ counts, int src_bits, int val_bits, const float* __restrict__ dinv,
                  int32_t* __restrict__ col_idx, float* __restrict__ edge_w, int32_t* __restrict__ perm, int64_t m)
 {
-    const int64_t k = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (k >= m || k >= counts->nnz) return;
-    const u64 word = __ldcs(keys + k);
-    const u64 key = word >> val_bits;
-    const int32_t s = (int32_t)(key & ((1ull << src_bits) - 1ull));
-    const int32_t d = (int32_t)(key >> src_bits);
-    __stcs(col_idx + k, s);
-    __stcs(edge_w + k, __ldg(dinv + s) * __ldg(dinv + d));
-    if (write_perm) __stcs(perm + k, vals ? __ldcs(vals + k) : (int32_t)(word & ((1ull << val_bits) - 1ull)) - 1);
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * kKeyItems) + threadIdx.x;
+    const int64_t nnz = counts->nnz;
+    u64 word[kKeyItems];
+#pragma unroll
+    for (int j = 0; j < kKeyItems; ++j) {
+        const int64_t k = base + j * kThreads;
+        word[j] = (k < m && k < nnz) ? __ldcs(keys + k) : 0ull;
+    }
+    float ws[kKeyItems], wd[kKeyItems];
+#pragma unroll
+    for (int j = 0; j < kKeyItems; ++j) {
+        const u64 key = word[j] >> val_bits;
+        ws[j] = __ldg(dinv + (int32_t)(key & ((1ull << src_bits) - 1ull)));       // 0 for the padding words: in range
+        wd[j] = __ldg(dinv + (int32_t)(key >> src_bits));
+    }
+#pragma unroll
+    for (int j = 0; j < kKeyItems; ++j) {
+        const int64_t k = base + j * kThreads;
+        if (k >= m || k >= nnz) continue;
+        const u64 key = word[j] >> val_bits;
+        __stcs(col_idx + k, (int32_t)(key & ((1ull << src_bits) - 1ull)));
+        __stcs(edge_w + k, ws[j] * wd[j]);
+        if (write_perm) __stcs(perm + k, vals ? __ldcs(vals + k) : (int32_t)(word[j] & ((1ull << val_bits) - 1ull)) - 1);
+    }
 }
 
 // segments per hub row; entry n_hub (one past the end) is 0 so that the scan yields the total
@@ -598,11 +645,11 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
     if (m > 0) {
         int32_t* key_vals = packed ? nullptr : vals;
         if (itype == GNNFD_I32)
-            GNNFD_LAUNCH("make_keys", s, make_keys<int32_t>, blocks_for(m, kThreads), kThreads, 0,
+            GNNFD_LAUNCH("make_keys", s, make_keys<int32_t>, blocks_for(m, kThreads * kKeyItems), kThreads, 0,
                          static_cast<const int32_t*>(d_src), static_cast<const int32_t*>(d_dst), n, e, m, flags, L.src_bits,
                          vb, keys, key_vals, P.counts);
         else
-            GNNFD_LAUNCH("make_keys", s, make_keys<long long>, blocks_for(m, kThreads), kThreads, 0,
+            GNNFD_LAUNCH("make_keys", s, make_keys<long long>, blocks_for(m, kThreads * kKeyItems), kThreads, 0,
                          static_cast<const long long*>(d_src), static_cast<const long long*>(d_dst), n, e, m, flags,
                          L.src_bits, vb, keys, key_vals, P.counts);
         const int mask = (1 << L.digit_bits) - 1;
@@ -639,7 +686,7 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
     GNNFD_LAUNCH("degrees_and_classes", s, degrees_and_classes, blocks_for((size_t)n, kThreads), kThreads, 0, P.row_ptr, n,
                  P.dinv, P.rdeg, keys_alt, vals_alt, P.counts);
     if (m > 0)
-        GNNFD_LAUNCH("finalize_entries", s, finalize_entries, blocks_for(m, kThreads), kThreads, 0, keys,
+        GNNFD_LAUNCH("finalize_entries", s, finalize_entries, blocks_for(m, kThreads * kKeyItems), kThreads, 0, keys,
                      packed ? (const int32_t*)nullptr : (const int32_t*)vals, dedup ? 0 : 1, P.counts, L.src_bits, vb,
                      P.dinv, P.col_idx, P.edge_w, P.perm, m);
     // row_order = rows sorted by degree class, ascending row id inside a class: one stable radix pass
