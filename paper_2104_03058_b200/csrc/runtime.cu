@@ -76,15 +76,31 @@ __device__ __forceinline__ int32_t block_exclusive_scan(int32_t v, int32_t* tota
     return warp_off + inc - v;
 }
 
+// the kScanItems values of one thread, with two 16-byte loads when the whole group exists and is aligned
+__device__ __forceinline__ void load_scan_items(const int32_t* in, size_t base, size_t count, bool vec, int32_t (&item)[kScanItems])
+{
+    static_assert(kScanItems == 8, "two 16-byte vectors per thread");
+    if (vec && base + kScanItems <= count) {
+        const int4 a = *reinterpret_cast<const int4*>(in + base), b = *reinterpret_cast<const int4*>(in + base + 4);
+        item[0] = a.x; item[1] = a.y; item[2] = a.z; item[3] = a.w;
+        item[4] = b.x; item[5] = b.y; item[6] = b.z; item[7] = b.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i) item[i] = base + i < count ? in[base + i] : 0;
+    }
+}
+
 __global__ void __launch_bounds__(kScanThreads) scan_tile_sums(const int32_t* __restrict__ in, size_t count,
                                                              int32_t* __restrict__ sums)
 {
     __shared__ int32_t smem[8];
     const size_t base = (size_t)blockIdx.x * kScanTile + (size_t)threadIdx.x * kScanItems;
+    const bool vec = (reinterpret_cast<uintptr_t>(in) & 15u) == 0;
+    int32_t item[kScanItems];
+    load_scan_items(in, base, count, vec, item);
     int32_t v = 0;
 #pragma unroll
-    for (int i = 0; i < kScanItems; ++i)
-        if (base + i < count) v += in[base + i];
+    for (int i = 0; i < kScanItems; ++i) v += item[i];
     int32_t total;
     block_exclusive_scan(v, &total, smem);
     if (threadIdx.x == 0) sums[blockIdx.x] = total;
@@ -95,19 +111,27 @@ __global__ void __launch_bounds__(kScanThreads) scan_tiles(const int32_t* in, in
 {
     __shared__ int32_t smem[8];
     const size_t base = (size_t)blockIdx.x * kScanTile + (size_t)threadIdx.x * kScanItems;
+    const bool vec = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
     int32_t item[kScanItems];
+    load_scan_items(in, base, count, vec, item);
     int32_t v = 0;
 #pragma unroll
-    for (int i = 0; i < kScanItems; ++i) {
-        item[i] = base + i < count ? in[base + i] : 0;
-        v += item[i];
-    }
+    for (int i = 0; i < kScanItems; ++i) v += item[i];
     int32_t total;
     int32_t run = block_exclusive_scan(v, &total, smem) + (offsets ? offsets[blockIdx.x] : 0);
+    int32_t res[kScanItems];
 #pragma unroll
     for (int i = 0; i < kScanItems; ++i) {
-        if (base + i < count) out[base + i] = run;
+        res[i] = run;
         run += item[i];
+    }
+    if (vec && base + kScanItems <= count) {
+        *reinterpret_cast<int4*>(out + base) = make_int4(res[0], res[1], res[2], res[3]);
+        *reinterpret_cast<int4*>(out + base + 4) = make_int4(res[4], res[5], res[6], res[7]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i)
+            if (base + i < count) out[base + i] = res[i];
     }
 }
 
