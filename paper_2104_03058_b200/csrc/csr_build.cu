@@ -274,11 +274,22 @@ __device__ __forceinline__ uint32_t first_of_run_mask(const u64* __restrict__ ke
                                                       u64 (&word)[kUniqueItems])
 {
     u64 prev = first > 0 && first <= n_valid ? (__ldg(keys + first - 1) >> val_bits) : 0ull;
+    if (first + kUniqueItems <= n_valid) {            // whole group present: 16-byte loads (first is a multiple of 8)
+        const ulonglong2* k2 = reinterpret_cast<const ulonglong2*>(keys + first);
+#pragma unroll
+        for (int j = 0; j < kUniqueItems; j += 2) {
+            const ulonglong2 v = __ldcs(k2 + j / 2);
+            word[j] = v.x;
+            word[j + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < kUniqueItems; ++j) word[j] = first + j < n_valid ? __ldcs(keys + first + j) : 0ull;
+    }
     uint32_t mask = 0;
 #pragma unroll
     for (int j = 0; j < kUniqueItems; ++j) {
         const int64_t i = first + j;
-        word[j] = i < n_valid ? __ldcs(keys + i) : 0ull;
         const u64 key = word[j] >> val_bits;
         if (i < n_valid && (i == 0 || key != prev)) mask |= 1u << j;
         prev = key;
