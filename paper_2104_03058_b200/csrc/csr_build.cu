@@ -422,9 +422,16 @@ degrees_and_classes(const int32_t* __restrict__ row_ptr, int64_t n, float* __res
         const int c = __syncthreads_count(bin == b);
         if (threadIdx.x == 0 && c) atomicAdd(&counts->bin_count[b], c);
     }
+    // block maximum, then one atomic per block (every block updates the same word)
+    __shared__ int32_t warp_max[kThreads / 32];
+    deg = __reduce_max_sync(0xffffffffu, deg);
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = deg;
+    __syncthreads();
+    if (threadIdx.x == 0) {
 #pragma unroll
-    for (int o = 16; o; o >>= 1) deg = max(deg, __shfl_xor_sync(0xffffffffu, deg, o));
-    if ((threadIdx.x & 31) == 0 && deg > 0) atomicMax(&counts->max_degree, deg);
+        for (int w = 1; w < kThreads / 32; ++w) deg = max(deg, warp_max[w]);
+        if (deg > 0) atomicMax(&counts->max_degree, deg);
+    }
 }
 
 // col_idx, the GCN weight and (unless the duplicate removal already wrote it) perm of every slot
