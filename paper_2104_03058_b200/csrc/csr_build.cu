@@ -178,8 +178,23 @@ __device__ __forceinline__ int32_t block_scan(int32_t v, int32_t* total, int32_t
     return off + inc - v;
 }
 
+// Lanes of the warp that hold the same digit value (among the valid ones): one ballot per digit bit.
+// The match instruction gives the same mask, but measured on this part it occupies its pipe for about
+// 56 cycles per warp, against about 21 for the nine ballots and their masking.
+__device__ __forceinline__ unsigned lanes_with_equal_digit(int digit, bool valid)
+{
+    unsigned peers = __ballot_sync(0xffffffffu, valid);
+#pragma unroll
+    for (int b = 0; b < kMaxDigitBits; ++b) {
+        const bool bit = (digit >> b) & 1;
+        const unsigned with_bit = __ballot_sync(0xffffffffu, bit);
+        peers &= bit ? with_bit : ~with_bit;
+    }
+    return valid ? peers : 0u;
+}
+
 // Stable scatter of one tile.  A warp owns kWarpItems consecutive keys and walks them 32 at a time: keys
-// with equal digits inside a round are ranked by lane (match_any), across rounds by a per-warp running
+// with equal digits inside a round are ranked by lane (ballots over the digit's bits), across rounds by a per-warp running
 // count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
 // digit in shared memory and written out run by run, so that consecutive threads store to
 // consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
@@ -210,8 +225,8 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
 #pragma unroll
     for (int r = 0; r < kSortItems; ++r) {
         const bool valid = warp_base + r * 32 + lane < m;
-        const int digit = valid ? ((int)(key[r] >> shift) & mask) : kRadix;
-        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        const int digit = (int)(key[r] >> shift) & mask;
+        const unsigned peers = lanes_with_equal_digit(digit, valid);
         const int leader = __ffs(peers) - 1;
         // the leader of each digit bumps the warp's running count; a warp's shared-memory atomics on one
         // address complete in program order, so the rounds need no barrier between them
