@@ -180,7 +180,10 @@ __device__ __forceinline__ int32_t block_scan(int32_t v, int32_t* total, int32_t
 
 // Lanes of the warp that hold the same digit value (among the valid ones): one ballot per digit bit.
 // The match instruction gives the same mask, but measured on this part it occupies its pipe for about
-// 56 cycles per warp, against about 21 for the nine ballots and their masking.
+// 56 cycles per warp, against about 21 ALU cycles for the nine ballots and their masking.  The two run
+// on different pipes, so the scatter uses the match instruction for GNNFD_SCATTER_MATCH_ROUNDS of a
+// warp's 16 rounds and ballots for the rest (config 4, per build: all match 3.59 ms, all ballots 3.09,
+// 3 / 5 / 7 rounds of match 3.02 / 2.86 / 2.99).
 __device__ __forceinline__ unsigned lanes_with_equal_digit(int digit, bool valid)
 {
     unsigned peers = __ballot_sync(0xffffffffu, valid);
@@ -198,6 +201,9 @@ __device__ __forceinline__ unsigned lanes_with_equal_digit(int digit, bool valid
 // count, across warps by a prefix over the per-warp counts.  The tile is then laid out sorted by
 // digit in shared memory and written out run by run, so that consecutive threads store to
 // consecutive addresses; the run of digit d starts at the scanned histogram entry of (d, tile).
+#ifndef GNNFD_SCATTER_MATCH_ROUNDS
+#define GNNFD_SCATTER_MATCH_ROUNDS 5
+#endif
 #ifndef GNNFD_SCATTER_MIN_BLOCKS
 #define GNNFD_SCATTER_MIN_BLOCKS 3
 #endif
@@ -226,7 +232,9 @@ radix_scatter(const u64* __restrict__ keys_in, const int32_t* __restrict__ vals_
     for (int r = 0; r < kSortItems; ++r) {
         const bool valid = warp_base + r * 32 + lane < m;
         const int digit = (int)(key[r] >> shift) & mask;
-        const unsigned peers = lanes_with_equal_digit(digit, valid);
+        // some rounds use the match instruction, the others ballots: the two run on different pipes
+        const unsigned peers = r < GNNFD_SCATTER_MATCH_ROUNDS ? __match_any_sync(0xffffffffu, valid ? digit : kRadix)
+                                                              : lanes_with_equal_digit(digit, valid);
         const int leader = __ffs(peers) - 1;
         // the leader of each digit bumps the warp's running count; a warp's shared-memory atomics on one
         // address complete in program order, so the rounds need no barrier between them
