@@ -49,10 +49,42 @@ constexpr int kStageSlots = kLoads * 32;      // column indices (and weights) a 
 // r*S + t*EP + g (r = s / LPR, t = s % LPR), read back as a broadcast.  A lane covers VPL vectors of the
 // chunk (columns c + q*LPR, q < VPL, in vector units) so that the index traffic, the address
 // arithmetic and the shuffles are paid once per VPL * 16 gathered bytes.
+// The thread's second-level sums live in shared memory as tot_s[k][thread]; with a multiple of four sums
+// they are moved four at a time (tot_s is then indexed as float4 rows of the same array).
+template <int NV, bool ZERO_ACC>
+__device__ __forceinline__ void second_level(float (*tot_s)[kBlock], int tid, float* acc, int mode /*0 clear, 1 add acc, 2 fetch*/)
+{
+    if constexpr (NV % 4 == 0) {
+        float4* t4 = reinterpret_cast<float4*>(&tot_s[0][0]) + tid;          // element k4 of the thread: t4[k4 * kBlock]
+#pragma unroll
+        for (int k4 = 0; k4 < NV / 4; ++k4) {
+            float4& slot = t4[k4 * kBlock];
+            if (mode == 0) {
+                slot = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else if (mode == 1) {
+                float4 v = slot;
+                v.x += acc[4 * k4]; v.y += acc[4 * k4 + 1]; v.z += acc[4 * k4 + 2]; v.w += acc[4 * k4 + 3];
+                slot = v;
+                if (ZERO_ACC) acc[4 * k4] = acc[4 * k4 + 1] = acc[4 * k4 + 2] = acc[4 * k4 + 3] = 0.f;
+            } else {
+                const float4 v = slot;
+                acc[4 * k4] += v.x; acc[4 * k4 + 1] += v.y; acc[4 * k4 + 2] += v.z; acc[4 * k4 + 3] += v.w;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            if (mode == 0) tot_s[k][tid] = 0.f;
+            else if (mode == 1) { tot_s[k][tid] += acc[k]; if (ZERO_ACC) acc[k] = 0.f; }
+            else acc[k] += tot_s[k][tid];
+        }
+    }
+}
+
 template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, int EP>
 __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0,
                                             int chunk_end, int32_t (*stage_col)[kBlock / 32][kStageSlots],
-                                            float (*stage_w)[kBlock / 32][kStageSlots])
+                                            float (*stage_w)[kBlock / 32][kStageSlots], float (*tot_s)[kBlock])
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
@@ -93,6 +125,12 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         }
     }
 
+    // Two levels of accumulation: `acc` takes at most kChain products in a row, then moves into the
+    // thread's second-level sums (kept in shared memory, they cost no registers), so that no fp32 chain
+    // of a lane is longer than kChain + (entries of the lane) / kChain terms.  Long runs of equal-sign
+    // terms (a hub row fed by one source many times) otherwise drift by half an ulp per term.
+    constexpr int kChain = 64;
+    constexpr int FLUSH = SPB >= kChain ? 1 : kChain / SPB;      // batches between two moves
     float acc[VPL][VECN];
 #pragma unroll
     for (int q = 0; q < VPL; ++q)
@@ -101,6 +139,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 
     const uint32_t ld = (uint32_t)a.ldx;
     const int n_batches = __reduce_max_sync(kFull, (e - b + EPB - 1) / EPB);     // the warp loops together
+    const bool two_level = n_batches > FLUSH;                                    // short rows never leave the first level
+    if (two_level) second_level<VPL * VECN, true>(tot_s, tid, &acc[0][0], 0);
 
     int32_t ucur[R];
     float wcur[R];
@@ -174,7 +214,9 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         }
 #pragma unroll
         for (int r = 0; r < R; ++r) { ucur[r] = unext[r]; wcur[r] = wnext[r]; }
+        if (two_level && (ib + 1) % FLUSH == 0) second_level<VPL * VECN, true>(tot_s, tid, &acc[0][0], 1);
     }
+    if (two_level) second_level<VPL * VECN, true>(tot_s, tid, &acc[0][0], 2);
 
     // fixed-order combination of the EP partial sums of the row
 #pragma unroll
@@ -216,6 +258,7 @@ __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggreg
 {
     __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
     __shared__ float stage_w[2][kBlock / 32][kStageSlots];
+    __shared__ __align__(16) float tot_s[VPL * VECN][kBlock];   // second-level sums of every thread
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
     const int chunk = (int)(blockIdx.x / per_chunk);
     const int rem = (int)(blockIdx.x % per_chunk);
@@ -232,12 +275,12 @@ __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggreg
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
-        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
-        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
-        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
-        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
-        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end, stage_col, stage_w); break;
+        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
     }
 }
 
@@ -252,8 +295,13 @@ hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict__ hu
     if (i >= n_hub || j >= f) return;
     const int32_t row = row_order[hub_begin + i];
     const int32_t s0 = hub_seg_ptr[i], s1 = hub_seg_ptr[i + 1];
-    float acc = 0.f;
-    for (int32_t s = s0; s < s1; ++s) acc += partial[(int64_t)s * fpad + j];
+    // segment sums in ascending order, in runs of 32 so that a row of very many segments keeps short chains
+    float acc = 0.f, run = 0.f;
+    for (int32_t s = s0; s < s1; ++s) {
+        run += partial[(int64_t)s * fpad + j];
+        if (((s - s0) & 31) == 31) { acc += run; run = 0.f; }
+    }
+    acc += run;
     if (use_rdeg) acc *= rdeg[row];
     store_elem(out, out_bf16, (int64_t)row * ldo + j, acc);
 }

@@ -86,7 +86,7 @@ constexpr int kStageSlots = kLoads * 32;      // column indices a warp stages pe
 // covers VPL adjacent vectors, all inside one head, so it needs one logit per entry.
 template <typename T, int VECN, int LPR, int VPL, int EP>
 __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int block_in_range, int col0, int chunk_end,
-                                         int32_t (*stage_col)[kBlock / 32][kStageSlots])
+                                         int32_t (*stage_col)[kBlock / 32][kStageSlots], float (*tot_s)[kBlock])
 {
     constexpr int S = LPR * EP;
     constexpr int ROWS = kBlock / S;
@@ -135,14 +135,38 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
     const uint32_t ld = (uint32_t)a.ldz;
     const uint32_t heads = (uint32_t)a.heads;
 
-    float m = -CUDART_INF_F, l = 0.f;
+    // Two levels of accumulation (as in the GCN / SAGE gather): `acc` and `l` take at most kChain terms in a
+    // row, then move into the thread's second-level sums in shared memory (slot VPL * VECN holds the
+    // denominator).  The second level is expressed under its own maximum m_tot and is brought to the
+    // current one only when something is added to it.
+    constexpr int kChain = 64;
+    constexpr int FLUSH = SPB >= kChain ? 1 : kChain / SPB;
+    float m = -CUDART_INF_F, l = 0.f, m_tot = -CUDART_INF_F;
     float acc[VPL][VECN];
 #pragma unroll
     for (int q = 0; q < VPL; ++q)
 #pragma unroll
         for (int i = 0; i < VECN; ++i) acc[q][i] = 0.f;
+    auto move_to_second_level = [&]() {
+        const float sc = m_tot == -CUDART_INF_F ? 0.f : ex2(m_tot - m);     // m >= m_tot; both -inf before any entry
+        m_tot = m;
+        tot_s[VPL * VECN][tid] = fmaf(tot_s[VPL * VECN][tid], sc, l);
+        l = 0.f;
+#pragma unroll
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int i = 0; i < VECN; ++i) {
+                tot_s[q * VECN + i][tid] = fmaf(tot_s[q * VECN + i][tid], sc, acc[q][i]);
+                acc[q][i] = 0.f;
+            }
+    };
 
     const int n_batches = __reduce_max_sync(kFull, (e - b + EPB - 1) / EPB);
+    const bool two_level = n_batches > FLUSH;          // short rows never leave the first level
+    if (two_level) {
+#pragma unroll
+        for (int k = 0; k <= VPL * VECN; ++k) tot_s[k][tid] = 0.f;
+    }
     int32_t ucur[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -216,6 +240,15 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         else steps(std::false_type{});
 #pragma unroll
         for (int r = 0; r < R; ++r) ucur[r] = unext[r];
+        if (two_level && (ib + 1) % FLUSH == 0) move_to_second_level();
+    }
+    if (two_level) {
+        move_to_second_level();
+        l = tot_s[VPL * VECN][tid];
+#pragma unroll
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int i = 0; i < VECN; ++i) acc[q][i] = tot_s[q * VECN + i][tid];
     }
 
     // merge the EP groups of the row, fixed tree
@@ -269,6 +302,7 @@ template <typename T, int VECN, int LPR, int VPL>
 __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ GatArgs a)
 {
     __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
+    __shared__ float tot_s[VPL * VECN + 1][kBlock];        // second-level sums and denominator, one column per thread
     const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
     const int chunk = (int)(blockIdx.x / per_chunk);
     const int rem = (int)(blockIdx.x % per_chunk);
@@ -285,12 +319,12 @@ __global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ 
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gat_rows<T, VECN, LPR, VPL, 1>(a, rg, bir, col0, chunk_end, stage_col); break;
-        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, VPL, 2>(a, rg, bir, col0, chunk_end, stage_col); break;
-        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, VPL, 4>(a, rg, bir, col0, chunk_end, stage_col); break;
-        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, VPL, 8>(a, rg, bir, col0, chunk_end, stage_col); break;
-        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, VPL, 16>(a, rg, bir, col0, chunk_end, stage_col); break;
-        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, VPL, 32>(a, rg, bir, col0, chunk_end, stage_col); break;
+        case 0: gat_rows<T, VECN, LPR, VPL, 1>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
+        case 1: if constexpr (LPR * 2 <= 32) gat_rows<T, VECN, LPR, VPL, 2>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
+        case 2: if constexpr (LPR * 4 <= 32) gat_rows<T, VECN, LPR, VPL, 4>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
+        case 3: if constexpr (LPR * 8 <= 32) gat_rows<T, VECN, LPR, VPL, 8>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
+        case 4: if constexpr (LPR * 16 <= 32) gat_rows<T, VECN, LPR, VPL, 16>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
+        default: if constexpr (LPR == 1) gat_rows<T, VECN, LPR, VPL, 32>(a, rg, bir, col0, chunk_end, stage_col, tot_s); break;
     }
 }
 
@@ -321,13 +355,19 @@ gat_hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict_
 #pragma unroll
     for (int w = 0; w < kReduceWays; ++w) mx = fmaxf(mx, s_max[w][c]);
     float num = 0.f, den = 0.f;
-    if (ok)
+    if (ok) {
+        float num_run = 0.f, den_run = 0.f;
+        int in_run = 0;
         for (int32_t s = s0 + q; s < s1; s += kReduceWays) {
             const float* ml = partial_ml + ((int64_t)s * heads + h) * 2;
             const float w = merge_scale(ml[0], mx);
-            den = fmaf(ml[1], w, den);
-            num = fmaf(partial[(int64_t)s * fpad + j], w, num);
+            den_run = fmaf(ml[1], w, den_run);
+            num_run = fmaf(partial[(int64_t)s * fpad + j], w, num_run);
+            if (++in_run == 32) { num += num_run; den += den_run; num_run = den_run = 0.f; in_run = 0; }   // short chains
         }
+        num += num_run;
+        den += den_run;
+    }
     s_num[q][c] = num;
     s_den[q][c] = den;
     __syncthreads();

@@ -464,3 +464,29 @@ def test_random_row_read_measurement(g):
     assert err.value.status == g.WORKSPACE_TOO_SMALL
     with pytest.raises(g.GnnfdError):
         g.measure_random_row_reads(buf, rows=16, pitch_bytes=128)
+
+
+@pytest.mark.parametrize("f,width", [(64, 64), (130, 128), (20, 5), (8, 8)])
+def test_long_runs_of_equal_terms_stay_inside_the_tolerance(g, f, width):
+    """A hub row fed thousands of times by the same source with same-sign features: every addition of a
+    plain fp32 chain then rounds in the same direction, so the error grows with the chain length.  The
+    kernels sum in two levels; the row must still meet the per-element bound."""
+    n, e = 3000, 60_000
+    rng = np.random.default_rng(f)
+    src = rng.integers(0, n, size=e).astype(np.int32)
+    dst = rng.integers(0, n, size=e).astype(np.int32)
+    dst[: e // 2] = 7                      # one row of ~30,000 entries ...
+    src[: e // 3] = 11                     # ... two thirds of them copies of one edge
+    x = (np.abs(gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=f)) + 0.5).astype(np.float32)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, 0)
+    csr = g.build_csr(n, dev(src), dev(dst), 0)
+    for model, fn in (("gcn", g.aggregate_gcn), ("sage", g.aggregate_sage)):
+        want, scale = orc.aggregate(model, row_ptr, col, x, f)
+        assert_close_f32(fn(csr, dev(x), f=f, chunk_width=width).cpu().numpy(), want, scale, "%s f %d" % (model, f))
+    if f % 8 == 0:
+        heads, dim = f // 8, 8
+        a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.2, seed=f, stream=5)
+        a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.2, seed=f, stream=6)
+        want, scale = orc.aggregate_gat(row_ptr, col, x, a_src, a_dst, heads, dim, 0.2)
+        got = g.aggregate_gat(csr, dev(x), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
+        assert_close_f32(got.cpu().numpy(), want, scale, "gat f %d" % f)
