@@ -333,11 +333,13 @@ __global__ void __launch_bounds__(kBlock) edge_softmax_hub_merge(const __grid_co
     const int32_t s0 = a.hub_seg_ptr[i], s1 = a.hub_seg_ptr[i + 1];
     float m = -CUDART_INF_F;
     for (int32_t s = s0; s < s1; ++s) m = fmaxf(m, a.seg_stats[(int64_t)s * a.heads + h].x);
-    float l = 0.f;
+    float l = 0.f, run = 0.f;                      // runs of 32 segments: a row of very many segments keeps short chains
     for (int32_t s = s0; s < s1; ++s) {
         const float2 st = a.seg_stats[(int64_t)s * a.heads + h];
-        l += st.y * rescale(st.x, m);
+        run += st.y * rescale(st.x, m);
+        if (((s - s0) & 31) == 31) { l += run; run = 0.f; }
     }
+    l += run;
     const float2 row_stats = make_float2(m, 1.f / l);
     for (int32_t s = s0; s < s1; ++s) a.seg_stats[(int64_t)s * a.heads + h] = row_stats;
 }

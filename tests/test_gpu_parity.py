@@ -490,3 +490,31 @@ def test_long_runs_of_equal_terms_stay_inside_the_tolerance(g, f, width):
         want, scale = orc.aggregate_gat(row_ptr, col, x, a_src, a_dst, heads, dim, 0.2)
         got = g.aggregate_gat(csr, dev(x), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
         assert_close_f32(got.cpu().numpy(), want, scale, "gat f %d" % f)
+
+
+def test_one_row_of_two_million_entries(g):
+    """Nearly 2,000 hub segments in one row: the per-row merges of the segment results (sums, softmax
+    denominators) must not become long fp32 chains either."""
+    n, e, f = 100, 2_000_000, 8
+    rng = np.random.default_rng(5)
+    src = rng.integers(0, n, size=e).astype(np.int32)
+    dst = np.full(e, 7, np.int32)
+    dst[:1000] = rng.integers(0, n, size=1000)
+    x = (np.abs(gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=5)) + 0.5).astype(np.float32)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, 0)
+    csr = g.build_csr(n, dev(src), dev(dst), 0)
+    assert csr.max_degree > 1_990_000
+    for model, fn in (("gcn", g.aggregate_gcn), ("sage", g.aggregate_sage)):
+        want, scale = orc.aggregate(model, row_ptr, col, x, f)
+        assert_close_f32(fn(csr, dev(x), f=f, chunk_width=f).cpu().numpy(), want, scale, model)
+    a_src = gg.features_f32(1, f, dist="normal", p0=0, p1=0.2, seed=5, stream=5)
+    a_dst = gg.features_f32(1, f, dist="normal", p0=0, p1=0.2, seed=5, stream=6)
+    want, scale = orc.aggregate_gat(row_ptr, col, x, a_src, a_dst, 1, f, 0.2)
+    got = g.aggregate_gat(csr, dev(x), dev(a_src), dev(a_dst), 1, f, 0.2, chunk_width=f)
+    assert_close_f32(got.cpu().numpy(), want, scale, "gat")
+    s_src, s_dst = g.gat_scores(dev(x), dev(a_src), dev(a_dst), 1, f)
+    alpha = g.edge_softmax(csr, s_src, s_dst, 0.2).cpu().numpy()
+    want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), 0.2)
+    assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
+    sums = np.add.reduceat(alpha.astype(np.float64), row_ptr[:-1][np.diff(row_ptr) > 0], axis=0)
+    assert np.abs(sums - 1.0).max() <= 1e-5
