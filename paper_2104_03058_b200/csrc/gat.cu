@@ -28,7 +28,7 @@ struct GatArgs {
     float* partial_ml;   // [n_segments, heads, 2] running max and denominator of hub segments
     int64_t ldz, ldo;
     float slope;
-    int32_t f, heads, dim, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16;
+    int32_t f, heads, dim, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16, wide_ok;
     int32_t n_ranges;
     Range range[kMaxRanges];
 };
@@ -127,6 +127,8 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
             e = a.row_ptr[row + 1];
         }
     }
+    // one 32-byte load per entry when both vectors of the lane exist and every row start allows it
+    const bool wide = a.wide_ok && okq[VPL - 1];
     const float sd = active ? a.s_dst[(int64_t)row * a.heads + h] : 0.f;
     const float* ssrc = a.s_src + h;
     // logits are kept in base 2: LeakyReLU(x) * log2 e = c1 * x + c2 * |x|
@@ -202,10 +204,15 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
                     const uint32_t uu = FULL ? (uint32_t)u : (uint32_t)max(u, 0);
                     lg[i] = valid[i] ? __ldg(ssrc + (size_t)uu * heads) : 0.f;
                     const size_t off = (size_t)uu * ld;
+                    if (VPL == 2 && VECN * sizeof(T) == 16 && wide) {
+                        if (valid[i]) load_pair(v[i][0], v[i][VPL - 1], zq[0] + off);     // the lane's two vectors are adjacent
+                        else { v[i][0].zero(); v[i][VPL - 1].zero(); }
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < VPL; ++q) {
-                        if (valid[i]) v[i][q].load(zq[q] + off);
-                        else v[i][q].zero();
+                        for (int q = 0; q < VPL; ++q) {
+                            if (valid[i]) v[i][q].load(zq[q] + off);
+                            else v[i][q].zero();
+                        }
                     }
                 }
                 float mx = m;
@@ -500,6 +507,9 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     a.n_ctiles = (cw + lpr * vpl * elems - 1) / (lpr * vpl * elems);
     a.fpad = (int32_t)align_up((size_t)f, 4);
     a.out_bf16 = odt == GNNFD_BF16;
+    // 32-byte loads of a lane's vector pair need every pair to start on a 32-byte boundary
+    a.wide_ok = vec && vpl == 2 && ((uintptr_t)d_z % 32 == 0) && ((ldz * zsize) % 32 == 0) &&
+                (n_chunks == 1 || (cw * zsize) % 32 == 0);
 
     const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges);
     a.blocks_per_tile = (int32_t)blocks;
