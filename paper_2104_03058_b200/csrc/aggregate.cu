@@ -27,7 +27,7 @@ struct GatherArgs {
     void* out;
     float* partial;
     int64_t ldx, ldo;
-    int32_t f, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16, out_vec_ok;
+    int32_t f, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16, out_vec_ok, wide_ok;
     int32_t n_ranges;
     Range range[kMaxRanges];
 };
@@ -81,7 +81,7 @@ __device__ __forceinline__ void second_level(float (*tot_s)[kBlock], int tid, fl
     }
 }
 
-template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, int EP>
+template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, bool WIDE, int EP>
 __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0,
                                             int chunk_end, int32_t (*stage_col)[kBlock / 32][kStageSlots],
                                             float (*stage_w)[kBlock / 32][kStageSlots], float (*tot_s)[kBlock])
@@ -107,11 +107,13 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     const T* xq[VPL];
 #pragma unroll
     for (int q = 0; q < VPL; ++q) {
-        jq[q] = col0 + (c + q * LPR) * VECN;
+        // with 32-byte loads a lane's two vectors are neighbours, otherwise they lie LPR vectors apart
+        jq[q] = col0 + (WIDE ? c * VPL + q : c + q * LPR) * VECN;
         okq[q] = jq[q] < chunk_end;
         xq[q] = static_cast<const T*>(a.x) + (okq[q] ? jq[q] : col0);   // out-of-chunk lanes re-read a valid column
     }
 
+    const bool wide = WIDE && okq[VPL - 1];            // both vectors of the lane exist: one 32-byte load per entry
     int32_t row = 0, b = 0, e = 0;
     if (active) {
         if (rg.hub) {
@@ -185,8 +187,12 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
                     const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
                     if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)u * ld;
+                    if (WIDE && wide) {
+                        load_pair(v[i][0], v[i][VPL - 1], xq[0] + off);
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
+                        for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
+                    }
                 }
             } else {
 #pragma unroll
@@ -195,10 +201,15 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
                     const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
                     if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)max(u, 0) * ld;
+                    if (WIDE && wide) {
+                        if (u >= 0) load_pair(v[i][0], v[i][VPL - 1], xq[0] + off);
+                        else { v[i][0].zero(); v[i][VPL - 1].zero(); }
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < VPL; ++q) {
-                        if (u >= 0) v[i][q].load(xq[q] + off);
-                        else v[i][q].zero();
+                        for (int q = 0; q < VPL; ++q) {
+                            if (u >= 0) v[i][q].load(xq[q] + off);
+                            else v[i][q].zero();
+                        }
                     }
                 }
             }
@@ -253,7 +264,7 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     }
 }
 
-template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED>
+template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, bool WIDE = false>
 __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggregate(const __grid_constant__ GatherArgs a)
 {
     __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
@@ -275,12 +286,12 @@ __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggreg
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
     switch (rg.ep_log2) {
-        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
-        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
-        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 4>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
-        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 8>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
-        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 16>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
-        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, 32>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 2: if constexpr (LPR * 4 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 4>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 3: if constexpr (LPR * 8 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 8>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        case 4: if constexpr (LPR * 16 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 16>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
+        default: if constexpr (LPR == 1) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 32>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
     }
 }
 
@@ -311,9 +322,18 @@ hub_reduce(const int32_t* __restrict__ row_order, const int32_t* __restrict__ hu
 typedef void (*GatherKernel)(const GatherArgs);
 
 template <typename T, int VECN, bool WEIGHTED>
-static GatherKernel pick_lpr(int lpr, int vpl)
+static GatherKernel pick_lpr(int lpr, int vpl, bool wide)
 {
     if (vpl == 1) return gather_aggregate<T, VECN, 1, 1, WEIGHTED>;
+    if constexpr (VECN * sizeof(T) == 16) {
+        if (wide) {          // narrow chunks whose vector pairs start on 32-byte boundaries
+            switch (lpr) {
+                case 1: return gather_aggregate<T, VECN, 1, 2, WEIGHTED, true>;
+                case 2: return gather_aggregate<T, VECN, 2, 2, WEIGHTED, true>;
+                default: return gather_aggregate<T, VECN, 4, 2, WEIGHTED, true>;
+            }
+        }
+    }
     switch (lpr) {
         case 1: return gather_aggregate<T, VECN, 1, 2, WEIGHTED>;
         case 2: return gather_aggregate<T, VECN, 2, 2, WEIGHTED>;
@@ -325,10 +345,11 @@ static GatherKernel pick_lpr(int lpr, int vpl)
 }
 
 template <bool WEIGHTED>
-static GatherKernel pick_kernel(gnnfd_dtype_t xdt, bool vec, int lpr, int vpl)
+static GatherKernel pick_kernel(gnnfd_dtype_t xdt, bool vec, int lpr, int vpl, bool wide)
 {
-    if (xdt == GNNFD_F32) return vec ? pick_lpr<float, 4, WEIGHTED>(lpr, vpl) : pick_lpr<float, 1, WEIGHTED>(lpr, vpl);
-    return vec ? pick_lpr<__nv_bfloat16, 8, WEIGHTED>(lpr, vpl) : pick_lpr<__nv_bfloat16, 1, WEIGHTED>(lpr, vpl);
+    if (xdt == GNNFD_F32)
+        return vec ? pick_lpr<float, 4, WEIGHTED>(lpr, vpl, wide) : pick_lpr<float, 1, WEIGHTED>(lpr, vpl, false);
+    return vec ? pick_lpr<__nv_bfloat16, 8, WEIGHTED>(lpr, vpl, wide) : pick_lpr<__nv_bfloat16, 1, WEIGHTED>(lpr, vpl, false);
 }
 
 static size_t partial_bytes(const gnnfd_csr_t* csr, int32_t f)
@@ -369,6 +390,13 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
     a.n_ctiles = (cw + lpr * vpl * elems - 1) / (lpr * vpl * elems);
     a.fpad = (int32_t)align_up((size_t)f, 4);
     a.out_bf16 = odt == GNNFD_BF16;
+    // 32-byte loads of a lane's vector pair: every pair must start on a 32-byte boundary, and the chunk must
+    // be narrow (up to 128 bytes, four lanes per row).  There the pair load halves the cache lines an
+    // instruction touches (hidden width 8 / 16 / 32 on the config-4 graph: 0.84 / 1.04 / 1.28 -> 0.61 / 0.77 /
+    // 0.99 ms); with eight or more lanes per row the strided single vectors already cover whole lines and
+    // the pair form is slower (config 4 at 64 columns 16.2 -> 18.4 ms).
+    a.wide_ok = vec && vpl == 2 && lpr <= 4 && ((uintptr_t)d_x % 32 == 0) && ((ldx * xsize) % 32 == 0) &&
+                (n_chunks == 1 || (cw * xsize) % 32 == 0);
     a.out_vec_ok = odt == GNNFD_F32 && ((uintptr_t)d_out % 16 == 0) && (ldo % 4 == 0) && (n_chunks == 1 || cw % 4 == 0);
 
     const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges);
@@ -377,7 +405,7 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
     if (grid > 0x7fffffffll || blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
 
     if (grid > 0) {
-        GatherKernel kernel = weighted ? pick_kernel<true>(xdt, vec, lpr, vpl) : pick_kernel<false>(xdt, vec, lpr, vpl);
+        GatherKernel kernel = weighted ? pick_kernel<true>(xdt, vec, lpr, vpl, a.wide_ok != 0) : pick_kernel<false>(xdt, vec, lpr, vpl, a.wide_ok != 0);
         GNNFD_LAUNCH(weighted ? "gather_aggregate_gcn" : "gather_aggregate_sage", s, kernel, (unsigned)grid, kBlock, 0, a);
     }
     const int64_t n_hub = csr->bin_count[4];
