@@ -283,6 +283,9 @@ def test_config3_gat_and_edge_softmax(g):
     zz = np.abs(w.x.astype(np.float64)).reshape(w.n, w.heads, w.dim)
     s_scale = np.einsum("nhd,hd->nh", zz, np.abs(w.a_src.astype(np.float64)))
     assert_close_f32(s_src.cpu().numpy(), o_src, s_scale, "s_src")
+    d_scale = np.einsum("nhd,hd->nh", zz, np.abs(w.a_dst.astype(np.float64)))
+    assert_close_f32(s_dst.cpu().numpy(), o_dst, d_scale, "s_dst")
+    assert np.abs(o_src - o_dst).max() > 1e-2          # the two score sets differ, so a mix-up would show
     alpha = g.edge_softmax(csr, s_src, s_dst, w.negative_slope).cpu().numpy()
     want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), w.negative_slope)
     assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()

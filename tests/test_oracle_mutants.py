@@ -10,6 +10,16 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SOURCE = os.path.join(ROOT, "oracle", "oracle.cpp")
 
 MUTANTS = {
+    "gcn_tolerance_scale_inflated": ("                    aabs += std::fabs(m);\n                }\n                out[r * f + j] = acc;\n                if (abs_out) abs_out[r * f + j] = aabs;\n            }\n        }\n    }\n    return 0;\n}\n\n// GAT attention scores",
+                                     "                    aabs += 2.0 * std::fabs(m);\n                }\n                out[r * f + j] = acc;\n                if (abs_out) abs_out[r * f + j] = aabs;\n            }\n        }\n    }\n    return 0;\n}\n\n// GAT attention scores"),
+    "gat_tolerance_scale_inflated": ("                    const double m = a[k - b] * load_x(z, zdt, (int64_t)col_idx[k] * ldz + j);\n                    acc += m;\n                    aabs += std::fabs(m);",
+                                     "                    const double m = a[k - b] * load_x(z, zdt, (int64_t)col_idx[k] * ldz + j);\n                    acc += m;\n                    aabs += 100.0 * std::fabs(m);"),
+    "gat_tolerance_scale_runs_on_across_columns": ("                double acc = 0.0, aabs = 0.0;\n                for (int32_t k = b; k < e; ++k) {\n                    const double m = a[k - b]",
+                                                   "                double acc = 0.0; static thread_local double aabs = 0.0;\n                for (int32_t k = b; k < e; ++k) {\n                    const double m = a[k - b]"),
+    "fp32_score_wrapper_swaps_source_and_destination": ("return orc_edge_softmax(n, row_ptr, col_idx, a.data(), b.data(), heads, slope, alpha);",
+                                                        "return orc_edge_softmax(n, row_ptr, col_idx, b.data(), a.data(), heads, slope, alpha);"),
+    "fp32_score_wrapper_reuses_source_scores": ("for (size_t i = 0; i < a.size(); ++i) { a[i] = s_src[i]; b[i] = s_dst[i]; }",
+                                                "for (size_t i = 0; i < a.size(); ++i) { a[i] = s_src[i]; b[i] = s_src[i]; }"),
     "gcn_weight_uses_destination_twice": ("const double w = model == 0 ? dinv[u] * dinv[v] : rdeg;",
                                           "const double w = model == 0 ? dinv[v] * dinv[v] : rdeg;"),
     "csr_rows_by_source": ("edges.push_back({d, s, i});", "edges.push_back({s, d, i});"),

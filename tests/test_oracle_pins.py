@@ -45,12 +45,13 @@ def dense_sage(a, x):
     return (rdeg[:, None] * a) @ x
 
 
-def dense_gat(a, z, a_src, a_dst, heads, dim, slope):
+def dense_gat(a, z, a_src, a_dst, heads, dim, slope, with_abs=False):
     n = a.shape[0]
     zz = z.reshape(n, heads, dim)
     s_src = np.einsum("nhd,hd->nh", zz, a_src.astype(np.float64))
     s_dst = np.einsum("nhd,hd->nh", zz, a_dst.astype(np.float64))
     out = np.zeros((n, heads, dim))
+    out_abs = np.zeros((n, heads, dim))
     for h in range(heads):
         e = s_dst[:, h][:, None] + s_src[:, h][None, :]          # e[v, u]
         e = np.where(e >= 0, e, slope * e)
@@ -61,6 +62,9 @@ def dense_gat(a, z, a_src, a_dst, heads, dim, slope):
         den = p.sum(axis=1, keepdims=True)
         alpha = np.divide(p, den, out=np.zeros_like(p), where=den > 0)
         out[:, h, :] = alpha @ zz[:, h, :]
+        out_abs[:, h, :] = alpha @ np.abs(zz[:, h, :])
+    if with_abs:
+        return out.reshape(n, heads * dim), out_abs.reshape(n, heads * dim)
     return out.reshape(n, heads * dim)
 
 
@@ -81,6 +85,10 @@ def test_gcn_sage_match_dense_product(n, flags):
         want = dense(a, x.astype(np.float64))
         got, ab = orc.aggregate(model, row_ptr, col, x, 5)
         np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+        # the tolerance scale sum |w x| is the same product on absolute values (all weights are >= 0):
+        # pinned by equality, since every GPU bound is a multiple of it
+        want_ab = dense(a, np.abs(x.astype(np.float64)))
+        np.testing.assert_allclose(ab, want_ab, rtol=1e-12, atol=1e-13)
         assert (ab >= np.abs(got) - 1e-12).all()
 
 
@@ -95,9 +103,13 @@ def test_gat_matches_dense_masked_softmax(n, flags):
     a_dst = gg.features_f32(heads, dim, dist="normal", p0=0.0, p1=0.7, seed=n, stream=6)
     a = dense_adjacency(n, src, dst, flags)
     row_ptr, col, _ = orc.build_csr(n, src, dst, flags)
-    want = dense_gat(a, z.astype(np.float64), a_src, a_dst, heads, dim, 0.2)
-    got, _ = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2)
+    want, want_ab = dense_gat(a, z.astype(np.float64), a_src, a_dst, heads, dim, 0.2, with_abs=True)
+    got, ab = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2)
     np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(ab, want_ab, rtol=1e-12, atol=1e-13)       # the tolerance scale sum |alpha z|
+    for width in (1, 5, heads * dim):                                     # ... for every decomposition too
+        _, ab_w = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2, chunk_width=width)
+        np.testing.assert_array_equal(ab_w, ab)
     # alpha written out: rows sum to one, and alpha-weighted sum reproduces the aggregation
     s_src, s_dst = orc.gat_scores(z, a_src, a_dst, heads, dim)
     alpha = orc.edge_softmax(row_ptr, col, s_src, s_dst, 0.2)
@@ -110,6 +122,45 @@ def test_gat_matches_dense_masked_softmax(n, flags):
                                        rtol=1e-12, atol=1e-13)
         else:
             assert (got[v] == 0).all()
+
+
+def dense_alpha(a, s_src, s_dst, slope):
+    """alpha[v, u, h]: masked row softmax of LeakyReLU(s_src[u, h] + s_dst[v, h]) over the in-neighbours u of v;
+    multi-edges share the value (each copy is one softmax term, so the denominator counts it a[v, u] times)."""
+    e = s_dst[:, None, :] + s_src[None, :, :]
+    e = np.where(e >= 0, e, slope * e)
+    e = np.where(a[:, :, None] > 0, e, -np.inf)
+    m = e.max(axis=1, keepdims=True)
+    m = np.where(np.isfinite(m), m, 0.0)
+    p = np.exp(e - m)
+    den = (a[:, :, None] * p).sum(axis=1, keepdims=True)
+    return np.divide(p, den, out=np.zeros_like(p), where=den > 0)
+
+
+@pytest.mark.parametrize("n", [8, 33, 64])
+@pytest.mark.parametrize("flags", [0, SL, SY | DD | SL])
+def test_edge_softmax_with_fp32_scores_matches_dense_softmax(n, flags):
+    """The entry the GPU tests use: scores arrive as float32 (as the library's caller supplies them).  The
+    source and destination scores are drawn differently, so a wrapper that swaps or reuses them fails."""
+    heads = 3
+    src, dst = gg.uniform_graph(n, 4 * n, seed=3 * n + flags)
+    dst[dst == 2] = 0
+    s_src = gg.features_f32(n, heads, dist="normal", p0=0.5, p1=1.5, seed=n, stream=5)
+    s_dst = gg.features_f32(n, heads, dist="normal", p0=-1.0, p1=0.7, seed=n, stream=6)
+    assert s_src.dtype == np.float32 and s_dst.dtype == np.float32
+    a = dense_adjacency(n, src, dst, flags)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, flags)
+    got = orc.edge_softmax(row_ptr, col, s_src, s_dst, 0.2)
+    assert got.dtype == np.float64 and got.shape == (len(col), heads)
+    want = dense_alpha(a, s_src.astype(np.float64), s_dst.astype(np.float64), 0.2)
+    rows = np.repeat(np.arange(n), np.diff(row_ptr))
+    np.testing.assert_allclose(got, want[rows, col, :], rtol=1e-12, atol=1e-15)
+    # the float64 entry on the widened values is the same computation
+    np.testing.assert_array_equal(got, orc.edge_softmax(row_ptr, col, s_src.astype(np.float64),
+                                                        s_dst.astype(np.float64), 0.2))
+    # and it is not what the swapped scores give
+    swapped = orc.edge_softmax(row_ptr, col, s_dst, s_src, 0.2)
+    assert np.abs(swapped - got).max() > 1e-3
 
 
 # ------------------------------------------------------------------ CSR structure
