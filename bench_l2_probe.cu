@@ -1,12 +1,14 @@
-// Measurement aid: how fast this GPU serves random row reads out of a resident working set.  The
+// Helper of bench.py (not part of libgnnfd.so): how fast this GPU serves random row reads out of a resident working set.  The
 // gather kernels read rows of a chunk's slice in an order set by the graph; when the slice fits L2
 // their ceiling is what L2 delivers to the SMs for such reads, which no copy benchmark measures.
 // This kernel does only that: lanes in groups of eight read 256-byte rows (two 16-byte loads per
 // lane, eight rows in flight per group) whose numbers come from an integer hash, with no index stream,
 // no arithmetic worth the name and no output.
-#include "common.cuh"
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
 
-namespace gnnfd {
+namespace {
 
 constexpr int kProbeThreads = 256;
 constexpr int kProbeLanes = 8;          // lanes per row
@@ -45,42 +47,42 @@ random_row_reads(const float4* __restrict__ buf, uint32_t rows, uint32_t pitch_v
     if (sink && acc.x + acc.y + acc.z + acc.w == 1.2345e-30f) sink[0] = acc.x;      // keeps the loads alive
 }
 
-}  // namespace gnnfd
+}  // namespace
 
-extern "C" int gnnfd_measure_random_row_reads(const void* d_buf, size_t buf_bytes, int64_t rows, int64_t pitch_bytes,
+// Returns 0 on success, -1 for bad arguments, -4 when the buffer is too small, -6 on a CUDA error.
+extern "C" int bench_random_row_reads(const void* d_buf, size_t buf_bytes, int64_t rows, int64_t pitch_bytes,
                                               void* stream, double* gb_per_s)
 {
-    using namespace gnnfd;
     if (!d_buf || !gb_per_s || rows <= 0 || rows > 0x7fffffffll || pitch_bytes < kProbeRowBytes || pitch_bytes % 16 != 0 ||
         ((uintptr_t)d_buf & 15u))
-        return GNNFD_INVALID_ARG;
-    if ((size_t)rows * (size_t)pitch_bytes > buf_bytes) return GNNFD_WORKSPACE_TOO_SMALL;
+        return -1;
+    if ((size_t)rows * (size_t)pitch_bytes > buf_bytes) return -4;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int sms = 0, dev = 0;
-    GNNFD_CUDA_CHECK(cudaGetDevice(&dev));
-    GNNFD_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (cudaGetDevice(&dev) != cudaSuccess) return -6;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -6;
     const unsigned grid = (unsigned)(sms * 3);
     const int rounds = 2000;
     cudaEvent_t e0, e1;
-    GNNFD_CUDA_CHECK(cudaEventCreate(&e0));
-    GNNFD_CUDA_CHECK(cudaEventCreate(&e1));
+    if (cudaEventCreate(&e0) != cudaSuccess) return -6;
+    if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return -6; }
     float best = 0.f;
-    int rc = GNNFD_OK;
-    for (int rep = 0; rep < 4 && rc == GNNFD_OK; ++rep) {            // the first launch warms the working set
+    int rc = 0;
+    for (int rep = 0; rep < 4 && rc == 0; ++rep) {            // the first launch warms the working set
         cudaEventRecord(e0, s);
-        GNNFD_LAUNCH("random_row_reads", s, random_row_reads, grid, kProbeThreads, 0, static_cast<const float4*>(d_buf),
-                     (uint32_t)rows, (uint32_t)(pitch_bytes / 16), rounds, (float*)nullptr);
+        random_row_reads<<<grid, kProbeThreads, 0, s>>>(static_cast<const float4*>(d_buf), (uint32_t)rows,
+                                                        (uint32_t)(pitch_bytes / 16), rounds, (float*)nullptr);
         cudaEventRecord(e1, s);
         float ms = 0.f;
         cudaError_t err = cudaEventSynchronize(e1);
         if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
-        if (err != cudaSuccess) { set_cuda_error(err); rc = GNNFD_CUDA_ERROR; break; }
+        if (err != cudaSuccess) { rc = -6; break; }
         if (rep > 0 && (best == 0.f || ms < best)) best = ms;
     }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
-    if (rc != GNNFD_OK) return rc;
+    if (rc != 0) return rc;
     const double bytes = (double)grid * kProbeThreads / kProbeLanes * rounds * kProbeRowsInFlight * (double)kProbeRowBytes;
     *gb_per_s = bytes / (best * 1e-3) / 1e9;
-    return GNNFD_OK;
+    return 0;
 }

@@ -95,7 +95,9 @@ int gnnfd_csr_info(const gnnfd_csr_t* csr, int64_t* n, int64_t* nnz, const int32
                    const int32_t** d_col_idx, const int32_t** d_perm, const float** d_dinv_sqrt,
                    const float** d_rdeg, const float** d_edge_weight, int32_t* max_degree);
 
-/* The launch schedule.  bin_count[5]: rows with degree <= 8, <= 32, <= 128, <= GNNFD_HUB_DEGREE, and
+/* The launch schedule.  (The paper has no counterpart: its CPU scatter walks the edge list as it comes.
+ * This is how the library balances power-law rows over the GPU; exposed for inspection and tests.)
+ * bin_count[5]: rows with degree <= 8, <= 32, <= 128, <= GNNFD_HUB_DEGREE, and
  * hub rows.  d_row_order[n]: row ids sorted by degree class, ascending id inside a class; a class is
  * the exact degree up to 8, then a quarter octave of (degree - 1) up to GNNFD_HUB_DEGREE, then one
  * class for all hub rows, so every bin is a contiguous range and neighbouring rows have near-equal
@@ -160,9 +162,13 @@ int gnnfd_tune_chunk_width(const gnnfd_csr_t* csr, int model, const void* d_x, i
  * buffer to hand over.  Such a caller cannot obtain the hub-row workspace gnnfd_aggregate_gcn asks
  * for.  Here that workspace is a fixed array of GNNFD_STATIC_SCRATCH_BYTES inside the library image;
  * every device that loads the library carries it until the process exits.  The call itself performs
- * no cudaMalloc / cudaFree and calls no allocating routine.
+ * no cudaMalloc / cudaFree and calls no allocating routine -- with one exception: while the optional
+ * per-kernel timing is switched on (gnnfd_kernel_timing_enable(1), a diagnostic that is off by
+ * default) every launch of the library creates a pair of CUDA events, this entry point's included;
+ * leave the timing off where allocation is not allowed.
  *
- * Same arguments and same results (bit for bit) as gnnfd_aggregate_gcn, minus the scratch pair.
+ * Same arguments and same results (bit for bit: it runs the same kernels on the same data) as
+ * gnnfd_aggregate_gcn, minus the scratch pair.
  * Limits and rules:
  *   - returns GNNFD_STATIC_SCRATCH_EXCEEDED when gnnfd_aggregate_workspace_bytes(csr, f) is larger
  *     than GNNFD_STATIC_SCRATCH_BYTES (hub segments x f rounded up to 4, x 4 bytes); nothing is launched;
@@ -180,6 +186,14 @@ int gnnfd_aggregate_gcn_static(const gnnfd_csr_t* csr, const void* d_x, int64_t 
 
 /* ------------------------------------------------------------------ GAT
  *
+ * The attention aggregator is the third model the paper evaluates (Section II-A lists it with GCN and
+ * GraphSAGE as the message-passing models under study; Section III runs it with a decomposition
+ * granularity of 8 columns, one head, and studies that granularity against the hidden width).  The
+ * paper gives no formula; the definition below is the cited GAT model's, evaluated on the
+ * destination-indexed edge list as Section II-C describes the framework's chunked `propagate`: the
+ * attention coefficients belong to the Message step and depend on whole heads, the weighted sum is the
+ * Aggregate step and is what Algorithm 1 decomposes.
+ *
  * Scores (full head width, computed once, never per chunk):
  *   s_src[u, h] = sum_d a_src[h, d] * z[u, h*dim + d],   s_dst[v, h] likewise with a_dst.
  * Logit of CSR entry k of row v, head h: LeakyReLU(s_src[col_idx[k], h] + s_dst[v, h]) with the given
@@ -189,12 +203,17 @@ int gnnfd_aggregate_gcn_static(const gnnfd_csr_t* csr, const void* d_x, int64_t 
  * over the row; chunk_width decomposes the flattened heads*dim columns (column j uses head j / dim).
  */
 
-/* d_z [n, ldz] of zdt; d_a_src / d_a_dst [heads, dim] fp32; d_s_src / d_s_dst [n, heads] fp32 out. */
+/* The per-vertex halves of the attention logit (the linear part of the cited model's Message step,
+ * Section II-A), computed once per layer from the full head width.
+ * d_z [n, ldz] of zdt; d_a_src / d_a_dst [heads, dim] fp32; d_s_src / d_s_dst [n, heads] fp32 out. */
 int gnnfd_gat_scores(int64_t n, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
                      const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst,
                      void* stream);
 
-/* Scratch for gnnfd_aggregate_gat: the two score arrays plus hub-row partials. */
+/* Scratch for gnnfd_aggregate_gat: the two score arrays plus hub-row partials.
+ * gnnfd_aggregate_gat is Algorithm 1's loop over decomposition layers for the attention model: Message
+ * (coefficient times source feature) and Aggregate (sum over the row) per chunk of chunk_width columns,
+ * Concat by writing each chunk into its own output columns. */
 int gnnfd_gat_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, size_t* scratch_bytes);
 
 int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt,
@@ -202,7 +221,9 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
                         float negative_slope, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
                         int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
 
-/* Materialised edge softmax: alpha[k, h] for every CSR slot k, [nnz, heads] fp32 in CSR order, from
+/* Materialised edge softmax (the normalisation inside the cited attention model's Message step,
+ * Section II-A, written out instead of fused; Section II-C's gather-scatter framework materialises it
+ * the same way): alpha[k, h] for every CSR slot k, [nnz, heads] fp32 in CSR order, from
  * caller-supplied scores d_s_src / d_s_dst [n, heads] fp32 (logit and softmax as defined above).
  * d_scratch: per-call buffer of gnnfd_edge_softmax_workspace_bytes(csr, heads) bytes (the running
  * maximum and sum of every hub-row segment; 0 bytes when the graph has no hub row, NULL is then
@@ -252,15 +273,6 @@ int64_t gnnfd_launch_count(void);
  * distinct kernels seen (may exceed capacity), or a negative status. */
 int gnnfd_kernel_timing_enable(int on);
 int gnnfd_kernel_timing_read(const char** names, double* ms, int64_t* launches, int capacity);
-
-/* Measurement aid for the roofline of the gather kernels (which are bound by L2-to-SM bandwidth when a
- * chunk's slice is resident, not by HBM): reads 256-byte rows, drawn uniformly at random by an integer
- * hash from `rows` rows that lie pitch_bytes apart in d_buf, with nothing else going on, and reports
- * the rate of the best of three timed launches in *gb_per_s.  d_buf is only read (any contents), must be
- * 16-byte aligned and hold rows * pitch_bytes bytes; pitch_bytes >= 256 and a multiple of 16.
- * Synchronises the stream. */
-int gnnfd_measure_random_row_reads(const void* d_buf, size_t buf_bytes, int64_t rows, int64_t pitch_bytes,
-                                   void* stream, double* gb_per_s);
 
 #ifdef __cplusplus
 }

@@ -64,7 +64,6 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_edge_softmax_workspace_bytes.argtypes = [vp, i32, pp(sz)]
         L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp, sz, vp]
         L.gnnfd_combine.argtypes = [i64, vp, i64, i32, i32, vp, i64, i32, vp, i64, i32, vp, vp]
-        L.gnnfd_measure_random_row_reads.argtypes = [vp, sz, i64, i64, vp, pp(ctypes.c_double)]
         L.gnnfd_status_string.argtypes = [ctypes.c_int]
         L.gnnfd_status_string.restype = ctypes.c_char_p
         L.gnnfd_last_cuda_error.restype = ctypes.c_int
@@ -100,9 +99,63 @@ def _matrix(t: torch.Tensor, cols: int, name: str):
     return ctypes.c_void_p(t.data_ptr()), t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
 
 
-def _alloc_bytes(nbytes: int, device) -> torch.Tensor:
-    # torch's caching allocator returns 512-byte aligned blocks
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+def _alloc_bytes(nbytes: int, device, stream=None) -> torch.Tensor:
+    """Scratch of at least `nbytes` (torch's caching allocator returns 512-byte aligned blocks).  The
+    block is taken under the stream the work will run on, so that the allocator does not hand it to
+    another stream's tensor while the kernels that use it are still queued."""
+    if stream is None:
+        return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    with torch.cuda.stream(stream):
+        return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def _same_device(csr_device, **tensors):
+    """Every operand must live on the device the CSR was built on (the library never migrates data)."""
+    for name, t in tensors.items():
+        if t is not None and torch.device(t.device) != torch.device(csr_device):
+            raise ValueError("%s is on %s but the CSR is on %s" % (name, t.device, csr_device))
+
+
+def _need_rows(t, rows: int, name: str):
+    if t.shape[0] < rows:
+        raise ValueError("%s has %d rows, the graph needs %d" % (name, t.shape[0], rows))
+
+
+def _extent(t):
+    """[first byte, one past the last byte) of the storage a strided 2-D / 1-D tensor touches."""
+    if t.numel() == 0:
+        return (t.data_ptr(), t.data_ptr())
+    last = sum((n - 1) * st for n, st in zip(t.shape, t.stride()))
+    return (t.data_ptr(), t.data_ptr() + (last + 1) * t.element_size())
+
+
+def _no_overlap(a, b, name_a: str, name_b: str):
+    """The kernels read features through the read-only data path, so an output that overlaps an input
+    is undefined behaviour the header forbids: refuse it here."""
+    a0, a1 = _extent(a)
+    b0, b1 = _extent(b)
+    if not (a0 < b1 and b0 < a1):
+        return
+    # Two column ranges of one row-major buffer interleave row by row without sharing an element: same row
+    # pitch, and the column intervals (taken modulo the pitch) apart.
+    if a.dim() == 2 and b.dim() == 2 and a.shape[0] > 1 and b.shape[0] > 1:
+        pitch_a, pitch_b = a.stride(0) * a.element_size(), b.stride(0) * b.element_size()
+        if pitch_a == pitch_b and pitch_a > 0:
+            first, second = (a, b) if a0 <= b0 else (b, a)
+            off = (max(a0, b0) - min(a0, b0)) % pitch_a
+            w_first = first.shape[1] * first.element_size()
+            w_second = second.shape[1] * second.element_size()
+            if w_first <= off and off + w_second <= pitch_a:
+                return
+    raise ValueError("%s and %s overlap in memory" % (name_a, name_b))
+
+
+def _check_aggregate_operands(csr, x, out, f: int, name_x: str = "x"):
+    """Shape, device and aliasing rules of the aggregation entry points, checked before any launch."""
+    _same_device(csr.device, **{name_x: x, "out": out})
+    _need_rows(x, csr.n, name_x)
+    _need_rows(out, csr.n, "out")
+    _no_overlap(x, out, name_x, "out")
 
 
 class Csr:
@@ -207,9 +260,11 @@ def _aggregate(fn, name, csr: Csr, x, f, chunk_width, out, out_dtype, scratch, s
         out = torch.empty((csr.n, f), dtype=out_dtype or torch.float32, device=x.device)
     xp, ldx = _matrix(x, f, "x")
     op, ldo = _matrix(out, f, "out")
+    _check_aggregate_operands(csr, x, out, f)
     need = aggregate_workspace_bytes(csr, f)
     if scratch is None and need:
-        scratch = _alloc_bytes(need, x.device)
+        scratch = _alloc_bytes(need, x.device, stream)
+    _same_device(csr.device, scratch=scratch)
     sp = ctypes.c_void_p(scratch.data_ptr()) if scratch is not None else None
     sn = scratch.numel() * scratch.element_size() if scratch is not None else 0
     _check(fn(csr.handle, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f, chunk_width, sp, sn,
@@ -246,9 +301,11 @@ def tune_chunk_width(csr: Csr, x: torch.Tensor, model: str = "gcn", f: int | Non
         out = torch.empty((csr.n, f), dtype=torch.float32, device=x.device)
     xp, ldx = _matrix(x, f, "x")
     op, ldo = _matrix(out, f, "out")
+    _check_aggregate_operands(csr, x, out, f)
     need = aggregate_workspace_bytes(csr, f)
     if scratch is None and need:
-        scratch = _alloc_bytes(need, x.device)
+        scratch = _alloc_bytes(need, x.device, stream)
+    _same_device(csr.device, scratch=scratch)
     sp = ctypes.c_void_p(scratch.data_ptr()) if scratch is not None else None
     sn = scratch.numel() * scratch.element_size() if scratch is not None else 0
     arr = (ctypes.c_int32 * len(candidates))(*candidates)
@@ -271,16 +328,30 @@ def aggregate_gcn_static(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_
         out = torch.empty((csr.n, f), dtype=torch.float32, device=x.device)
     xp, ldx = _matrix(x, f, "x")
     op, ldo = _matrix(out, f, "out")
+    _check_aggregate_operands(csr, x, out, f)
     _check(lib().gnnfd_aggregate_gcn_static(csr.handle, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f,
                                             chunk_width, _stream_ptr(stream)), "gnnfd_aggregate_gcn_static")
     return out
 
 
+def _attention_vectors(a_src, a_dst, heads: int, dim: int, device, stream):
+    """The two [heads, dim] fp32 attention vectors, contiguous and on `device`.  A conversion makes a
+    temporary; it is created under the launch stream for the same reason as the scratch buffers."""
+    for name, a in (("a_src", a_src), ("a_dst", a_dst)):
+        if a.numel() != heads * dim:
+            raise ValueError("%s must hold heads*dim = %d values" % (name, heads * dim))
+        if torch.device(a.device) != torch.device(device):
+            raise ValueError("%s is on %s, the features are on %s" % (name, a.device, device))
+    if stream is None:
+        return a_src.contiguous().float(), a_dst.contiguous().float()
+    with torch.cuda.stream(stream):
+        return a_src.contiguous().float(), a_dst.contiguous().float()
+
+
 def gat_scores(z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.Tensor, heads: int, dim: int, stream=None):
     n = z.shape[0]
     zp, ldz = _matrix(z, heads * dim, "z")
-    a_src = a_src.contiguous().float()
-    a_dst = a_dst.contiguous().float()
+    a_src, a_dst = _attention_vectors(a_src, a_dst, heads, dim, z.device, stream)
     s_src = torch.empty((n, heads), dtype=torch.float32, device=z.device)
     s_dst = torch.empty((n, heads), dtype=torch.float32, device=z.device)
     _check(lib().gnnfd_gat_scores(n, zp, ldz, _dtype_code(z), ctypes.c_void_p(a_src.data_ptr()),
@@ -304,10 +375,11 @@ def aggregate_gat(csr: Csr, z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.T
         out = torch.empty((csr.n, f), dtype=out_dtype or torch.float32, device=z.device)
     zp, ldz = _matrix(z, f, "z")
     op, ldo = _matrix(out, f, "out")
-    a_src = a_src.contiguous().float()
-    a_dst = a_dst.contiguous().float()
+    _check_aggregate_operands(csr, z, out, f, "z")
+    a_src, a_dst = _attention_vectors(a_src, a_dst, heads, dim, z.device, stream)
     if scratch is None:
-        scratch = _alloc_bytes(gat_workspace_bytes(csr, heads, dim), z.device)
+        scratch = _alloc_bytes(gat_workspace_bytes(csr, heads, dim), z.device, stream)
+    _same_device(csr.device, scratch=scratch)
     _check(lib().gnnfd_aggregate_gat(csr.handle, zp, ldz, _dtype_code(z), ctypes.c_void_p(a_src.data_ptr()),
                                      ctypes.c_void_p(a_dst.data_ptr()), heads, dim, negative_slope, op, ldo,
                                      _dtype_code(out), chunk_width, ctypes.c_void_p(scratch.data_ptr()),
@@ -326,14 +398,23 @@ def edge_softmax_workspace_bytes(csr: Csr, heads: int) -> int:
 def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_slope: float = 0.2,
                  out: torch.Tensor | None = None, scratch=None, stream=None) -> torch.Tensor:
     heads = s_src.shape[1]
-    s_src = s_src.contiguous()
-    s_dst = s_dst.contiguous()
+    if not (s_src.is_contiguous() and s_dst.is_contiguous()):
+        raise ValueError("scores must be contiguous")
     if s_src.dtype != torch.float32 or s_dst.dtype != torch.float32 or s_src.shape != s_dst.shape:
         raise TypeError("scores must be float32 [n, heads]")
+    if s_src.dim() != 2 or s_src.shape[0] != csr.n:
+        raise ValueError("scores must be [n, heads] with n = %d rows, got %s" % (csr.n, tuple(s_src.shape)))
     if out is None:
         out = torch.empty((csr.nnz, heads), dtype=torch.float32, device=s_src.device)
+    if out.dtype != torch.float32 or out.dim() != 2 or not out.is_contiguous() or out.shape[1] != heads \
+            or out.shape[0] < csr.nnz:
+        raise ValueError("alpha must be a contiguous float32 [nnz >= %d, heads = %d] tensor" % (csr.nnz, heads))
+    _same_device(csr.device, s_src=s_src, s_dst=s_dst, alpha=out)
+    _no_overlap(s_src, out, "s_src", "alpha")
+    _no_overlap(s_dst, out, "s_dst", "alpha")
     if scratch is None:
-        scratch = _alloc_bytes(edge_softmax_workspace_bytes(csr, heads), s_src.device)
+        scratch = _alloc_bytes(edge_softmax_workspace_bytes(csr, heads), s_src.device, stream)
+    _same_device(csr.device, scratch=scratch)
     _check(lib().gnnfd_edge_softmax(csr.handle, ctypes.c_void_p(s_src.data_ptr()), ctypes.c_void_p(s_dst.data_ptr()),
                                     heads, negative_slope, ctypes.c_void_p(out.data_ptr()),
                                     ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
@@ -356,19 +437,14 @@ def combine(x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, out: to
     xp, ldx = _matrix(x, f_in, "x")
     wp, ldw = _matrix(w_t, f_in, "w_t")
     op, ldo = _matrix(out, f_out, "out")
+    _same_device(x.device, w_t=w_t, out=out, status=status)
+    _need_rows(out, x.shape[0], "out")
+    _no_overlap(x, out, "x", "out")
+    _no_overlap(w_t, out, "w_t", "out")
     sp = ctypes.c_void_p(status.data_ptr()) if status is not None else None
     _check(lib().gnnfd_combine(x.shape[0], xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, op, ldo, _dtype_code(out), sp,
                                _stream_ptr(stream)), "gnnfd_combine")
     return out
-
-
-def measure_random_row_reads(buf: torch.Tensor, rows: int, pitch_bytes: int = 256, stream=None) -> float:
-    """gnnfd_measure_random_row_reads: GB/s at which random 256-byte rows of a resident set reach the SMs."""
-    out = ctypes.c_double()
-    _check(lib().gnnfd_measure_random_row_reads(ctypes.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size(), rows,
-                                                pitch_bytes, _stream_ptr(stream), ctypes.byref(out)),
-           "gnnfd_measure_random_row_reads")
-    return out.value
 
 
 def launch_count() -> int:

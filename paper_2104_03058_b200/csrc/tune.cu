@@ -1,6 +1,5 @@
 // Chunk-width selection by measurement.  The paper leaves the number of decomposition layers to the
-// user ("determined according to the memory capacity of the device and characteristics of datasets",
-// Section II-B); the best width depends on how the graph's gathers hit the caches, which a size
+// user, to be set from the device's memory and the dataset at hand (Section II-B); the best width depends on how the graph's gathers hit the caches, which a size
 // formula does not capture (an RMAT graph with 2 M vertices runs fastest undecomposed, the
 // Reddit-shaped graph at 64 columns), so the candidates are simply timed on the caller's data.
 #include "common.cuh"

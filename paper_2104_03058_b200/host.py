@@ -71,9 +71,12 @@ class HostPipeline:
             self.csr.destroy()
         self.csr = g.build_csr(self.n, self.d_src[slot][:e], self.d_dst[slot][:e], self.flags,
                                persistent=self.persistent, scratch=self.scratch)
-        if self.agg_scratch is None:
-            need = (g.gat_workspace_bytes(self.csr, self.heads, self.dim) if self.model == "gat"
-                    else g.aggregate_workspace_bytes(self.csr, self.f))
+        # the workspace depends on this graph's hub rows, so it is asked for per job and grown when needed
+        # (the old buffer may still be in use by the previous job's kernels on this stream: torch frees it
+        # in stream order)
+        need = (g.gat_workspace_bytes(self.csr, self.heads, self.dim) if self.model == "gat"
+                else g.aggregate_workspace_bytes(self.csr, self.f))
+        if self.agg_scratch is None or self.agg_scratch.numel() < need:
             self.agg_scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
         out = self.d_out[slot][:, :self.f]
         if self.model == "gat":
@@ -98,5 +101,3 @@ class HostPipeline:
         cur.wait_stream(self.s_in)
         cur.wait_stream(self.s_out)
 
-
-HostGcnPipeline = HostPipeline

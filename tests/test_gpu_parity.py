@@ -332,7 +332,7 @@ def test_gat_bf16_features(g):
 # ------------------------------------------------------------------ host-buffer front end
 
 def test_host_pipeline_matches_direct_calls(g):
-    from paper_2104_03058_b200.host import HostGcnPipeline
+    from paper_2104_03058_b200.host import HostPipeline
     n, f, ld = 3000, 20, 24
     jobs = []
     for seed in range(4):
@@ -341,7 +341,7 @@ def test_host_pipeline_matches_direct_calls(g):
         jobs.append((torch.from_numpy(src).pin_memory(), torch.from_numpy(dst).pin_memory(),
                      torch.from_numpy(x).pin_memory()))
     max_e = max(j[0].numel() for j in jobs)
-    pipe = HostGcnPipeline(n, max_e, f, ld, SL, 8)
+    pipe = HostPipeline(n, max_e, f, ld, SL, 8)
     outs = [torch.zeros((n, ld)).pin_memory() for _ in jobs]
     for i, job in enumerate(jobs):
         pipe.submit(*job, outs[i], next_job=jobs[i + 1] if i + 1 < len(jobs) else None)
@@ -351,6 +351,61 @@ def test_host_pipeline_matches_direct_calls(g):
         csr = g.build_csr(n, h_src.cuda(), h_dst.cuda(), SL)
         want = g.aggregate_gcn(csr, h_x.cuda(), f=f, chunk_width=8)
         assert torch.equal(out[:, :f], want.cpu())
+
+
+def test_host_pipeline_grows_its_workspace_for_a_graph_with_more_hub_rows(g):
+    from paper_2104_03058_b200.host import HostPipeline
+    n, f, e = 3000, 12, 40_000
+    jobs = []
+    for hubs in ((), (5,), (7, 1200, 2999)):                 # 0, 1 and 3 rows above the hub threshold
+        src, dst = gg.uniform_graph(n, e, seed=len(hubs))
+        for i, v in enumerate(hubs):
+            dst[i * 5000:(i + 1) * 5000] = v
+        x = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=len(hubs))
+        jobs.append((torch.from_numpy(src).pin_memory(), torch.from_numpy(dst).pin_memory(),
+                     torch.from_numpy(x).pin_memory()))
+    pipe = HostPipeline(n, e, f, f, 0, 4)
+    outs = [torch.zeros((n, f)).pin_memory() for _ in jobs]
+    for i, job in enumerate(jobs):
+        csr = pipe.submit(*job, outs[i])
+        assert csr.bin_count[4] == (0, 1, 3)[i]
+    pipe.finish()
+    torch.cuda.synchronize()
+    for (h_src, h_dst, h_x), out in zip(jobs, outs):
+        csr = g.build_csr(n, h_src.cuda(), h_dst.cuda(), 0)
+        assert torch.equal(out, g.aggregate_gcn(csr, h_x.cuda(), f=f, chunk_width=4).cpu())
+
+
+def test_binding_refuses_bad_operands_before_any_launch(g):
+    n, f = 500, 8
+    src, dst = gg.uniform_graph(n, 4000, seed=3)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    x = torch.zeros((n, f), device="cuda")
+    out = torch.zeros((n, f), device="cuda")
+    a = torch.zeros((2, 4), device="cuda")
+    s = torch.zeros((n, 2), device="cuda")
+    before = g.launch_count()
+    for call in (lambda: g.aggregate_gcn(csr, x[:n - 1], f=f, out=out),            # x too short
+                 lambda: g.aggregate_sage(csr, x, f=f, out=out[:10]),               # out too short
+                 lambda: g.aggregate_gcn(csr, x, f=f, out=x),                       # in place
+                 lambda: g.aggregate_gcn(csr, x.cpu(), f=f),                        # wrong device
+                 lambda: g.aggregate_gat(csr, x[:100], a, a, 2, 4, out=out),        # z too short
+                 lambda: g.aggregate_gat(csr, x, a[:1], a, 2, 4, out=out),          # attention vector too short
+                 lambda: g.edge_softmax(csr, s[:n - 3], s[:n - 3]),                 # scores too short
+                 lambda: g.edge_softmax(csr, s, s, out=torch.zeros((csr.nnz - 1, 2), device="cuda")),
+                 lambda: g.aggregate_gcn_static(csr, x[:n - 1], f=f, out=out)):
+        with pytest.raises(ValueError):
+            call()
+    assert g.launch_count() == before
+    # a non-default stream: scratch and temporaries are taken under that stream
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    x.normal_()
+    torch.cuda.synchronize()
+    want = g.aggregate_gcn(csr, x, f=f)
+    got = g.aggregate_gcn(csr, x, f=f, stream=side)
+    side.synchronize()
+    assert torch.equal(got, want)
 
 
 def test_chunk_width_tuner_picks_a_candidate_and_leaves_a_valid_result(g):
@@ -455,18 +510,6 @@ def test_csr_sort_boundaries(g, n, e, flags):
     assert torch.equal(csr.perm.cpu(), torch.from_numpy(perm))
     assert sum(csr.bin_count) == n
 
-
-def test_random_row_read_measurement(g):
-    buf = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
-    rate = g.measure_random_row_reads(buf, rows=(8 << 20) // 256, pitch_bytes=256)
-    assert rate > 100.0                                   # GB/s; any B200 is far above this
-    strided = g.measure_random_row_reads(buf, rows=(8 << 20) // 512, pitch_bytes=512)
-    assert strided > 100.0
-    with pytest.raises(g.GnnfdError) as err:              # more rows than the buffer holds
-        g.measure_random_row_reads(buf, rows=(8 << 20) // 256 + 1, pitch_bytes=256)
-    assert err.value.status == g.WORKSPACE_TOO_SMALL
-    with pytest.raises(g.GnnfdError):
-        g.measure_random_row_reads(buf, rows=16, pitch_bytes=128)
 
 
 @pytest.mark.parametrize("f,width", [(64, 64), (130, 128), (20, 5), (8, 8)])
