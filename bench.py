@@ -126,11 +126,11 @@ def make_workload(name: str, seed: int):
     return WORKLOADS[name][0](seed)
 
 
-def roofline_bytes(w, nnz: int) -> int:
+def roofline_bytes(w, nnz: int, f: int | None = None) -> int:
     """Algorithmic bytes of one aggregation launch: every row pointer once, the CSR column indices once,
     the GCN weights once, every gathered feature (and, for GAT, every gathered score)."""
     elem = 2 if w.dtype == "bf16" else 4
-    b = 4 * (w.n + 1) + 4 * nnz + nnz * w.f * elem
+    b = 4 * (w.n + 1) + 4 * nnz + nnz * (w.f if f is None else f) * elem
     if w.model == "gcn":
         b += 4 * nnz
     if w.model == "gat":
@@ -290,8 +290,12 @@ def run_ours(args):
         g.build.build_library()
     g.lib()
 
-    w = make_workload(args.workload, args.seed + rank)
+    # --shard columns: ONE graph for all ranks (same seed); each rank builds the CSR and aggregates only the
+    # decomposition layers of its column slab (strong scaling).  Default: an independent graph per rank (weak).
+    by_columns = args.shard == "columns"
+    w = make_workload(args.workload, args.seed + (0 if by_columns else rank))
     cw = args.chunk_width or WORKLOADS[args.workload][1]
+    j0, j1 = sharding.column_slab(w.f, cw, world, rank) if by_columns else (0, w.f)
     e = len(w.src)
     bf16 = w.dtype == "bf16"
     h_src = torch.from_numpy(w.src).pin_memory()
@@ -311,7 +315,13 @@ def run_ours(args):
     state = {"agg_scratch": None, "csr": None}
 
     def aggregate(csr, width):
-        if gat:
+        if by_columns:
+            sharding.aggregate_slab(csr, d_x, w.model, w.f, width, world, rank, out_view, a_src=a_src, a_dst=a_dst,
+                                    heads=w.heads, dim=w.dim, negative_slope=w.negative_slope,
+                                    scratch=state["agg_scratch"])
+            if args.gather and world > 1:
+                sharding.gather_slabs_(out_view, w.f, width)
+        elif gat:
             g.aggregate_gat(csr, d_x, a_src, a_dst, w.heads, w.dim, w.negative_slope, chunk_width=width, out=out_view,
                             scratch=state["agg_scratch"])
         elif w.model == "sage":
@@ -340,7 +350,7 @@ def run_ours(args):
     for _ in range(warmup):
         csr = step()
     nnz = csr.nnz
-    units_per_step = nnz * w.f
+    units_per_step = nnz * (j1 - j0)
 
     # ---- timed region: device-resident inputs
     sampler = ClockSampler(local_rank)
@@ -363,23 +373,44 @@ def run_ours(args):
 
     # ---- end to end: pinned host inputs in, result out, every step (the package's host-buffer front end:
     # double-buffered device copies, the next step's inputs and the previous result travel while the kernels run)
-    pipe = HostPipeline(w.n, e, w.f, w.ld, w.flags, cw, device=device, feature_dtype=h_x.dtype, model=w.model,
-                        heads=w.heads, dim=w.dim, a_src=a_src, a_dst=a_dst, negative_slope=w.negative_slope)
     job = (h_src, h_dst, h_x)
-    pipe.submit(*job, h_out)                         # warm-up job (allocates the aggregation workspace)
-    pipe.finish()
-    barrier()
-    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev2.record()
-    for i in range(args.steps):
-        pipe.submit(*job, h_out, next_job=job if i + 1 < args.steps else None)
-    pipe.finish()
-    ev3.record()
-    barrier()
-    ms_e2e = ev2.elapsed_time(ev3)
-    h2d = sum(t.numel() * t.element_size() for t in job)
-    d2h = h_out.numel() * 4
-    del pipe
+    if by_columns:
+        # a rank moves the edge list, its own columns of x in and its own columns of the result out
+        def e2e_step():
+            d_src.copy_(h_src, non_blocking=True)
+            d_dst.copy_(h_dst, non_blocking=True)
+            d_x[:, j0:j1].copy_(h_x[:, j0:j1], non_blocking=True)
+            step()
+            h_out[:, j0:j1].copy_(out[:, j0:j1], non_blocking=True)
+        e2e_step()
+        barrier()
+        ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev2.record()
+        for i in range(args.steps):
+            e2e_step()
+        ev3.record()
+        barrier()
+        ms_e2e = ev2.elapsed_time(ev3)
+        esize = h_x.element_size()
+        h2d = h_src.numel() * h_src.element_size() * 2 + w.n * (j1 - j0) * esize
+        d2h = w.n * (j1 - j0) * 4
+    else:
+        pipe = HostPipeline(w.n, e, w.f, w.ld, w.flags, cw, device=device, feature_dtype=h_x.dtype, model=w.model,
+                            heads=w.heads, dim=w.dim, a_src=a_src, a_dst=a_dst, negative_slope=w.negative_slope)
+        pipe.submit(*job, h_out)                         # warm-up job (allocates the aggregation workspace)
+        pipe.finish()
+        barrier()
+        ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev2.record()
+        for i in range(args.steps):
+            pipe.submit(*job, h_out, next_job=job if i + 1 < args.steps else None)
+        pipe.finish()
+        ev3.record()
+        barrier()
+        ms_e2e = ev2.elapsed_time(ev3)
+        h2d = sum(t.numel() * t.element_size() for t in job)
+        d2h = h_out.numel() * 4
+        del pipe
 
     # ---- aggregation alone (context for the step time), a few calls per chunk width
     agg_ms, agg_cold_ms = {}, {}
@@ -450,14 +481,20 @@ def run_ours(args):
     if slice_rows * 256 <= 0.6 * l2_bytes:
         l2_measured = measure_random_row_reads(out, slice_rows, 256)
 
+    rank_ms = ms
     ms, total_units = sharding.reduce_job_timing(ms, float(units_per_step), device=device)
     ms_e2e, _ = sharding.reduce_job_timing(ms_e2e, 0.0, device=device)
+    per_rank = [{"rank": rank, "columns": [j0, j1], "ms_per_step": rank_ms / args.steps}]
+    if world > 1:
+        gathered = [None] * world
+        dist.all_gather_object(gathered, per_rank[0])
+        per_rank = gathered
 
     if rank == 0:
         peak, peak_src = measured_peaks()
         name = KERNEL_OF_MODEL[w.model]
         k_ms, k_n = kernels.get(name, (0.0, 0))
-        bytes_launch = roofline_bytes(w, nnz)
+        bytes_launch = roofline_bytes(w, nnz, j1 - j0)
         achieved = bytes_launch / (k_ms / k_n * 1e-3) / 1e9 if k_n else None
         total_kernel_ms = sum(v[0] for v in kernels.values())
         x_mb = w.n * w.ld * (2 if bf16 else 4) // 2 ** 20
@@ -489,13 +526,17 @@ def run_ours(args):
         result = {
             "metric": METRIC, "value": total_units * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": warmup, "ms_per_step": ms / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "higher_is_better": True, "scaling": "strong" if by_columns else "weak", "vs_baseline": None,
             "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "description": WORKLOADS[args.workload][2],
                        "arithmetic": "fp32 multiply-add (bf16 features are widened exactly)" if bf16 else "fp32",
                        "step": "gnnfd_build_csr + gnnfd_aggregate_" + w.model, "n": w.n, "input_edges": e, "nnz": nnz,
                        "f": w.f, "feature_dtype": w.dtype, "chunk_width": cw,
-                       "parallelism": "independent graphs per GPU" if world > 1 else "1 GPU",
+                       "parallelism": ("feature-chunk slabs: one graph, CSR built on every GPU, each GPU aggregates "
+                                       "its chunk-aligned columns%s" % (", slabs all-gathered over NCCL" if args.gather
+                                                                        else ", no exchange")) if by_columns
+                       else ("independent graphs per GPU" if world > 1 else "1 GPU"),
+                       "ranks": per_rank,
                        "l2": "inputs vs the 126 MB L2: x %d MB, col_idx+weights %d MB per sweep (no flush between steps)"
                              % (x_mb, nnz * 8 // 2 ** 20)},
             "roofline": roofline,
@@ -562,6 +603,11 @@ def main():
     ap.add_argument("--sweep", type=int, nargs="*", default=[], help="extra chunk widths to time (aggregation only)")
     ap.add_argument("--combine-out", type=int, default=64,
                     help="output width of the dense transform timed beside the step (0: skip; fp32 workloads only)")
+    ap.add_argument("--shard", choices=["graphs", "columns"], default="graphs",
+                    help="graphs: every rank its own graph (weak scaling); columns: one graph, each rank aggregates the "
+                         "decomposition layers of its column slab (strong scaling)")
+    ap.add_argument("--gather", action="store_true",
+                    help="with --shard columns: all-gather the slabs (NCCL) so that every rank ends with the full result")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-rows", type=int, default=0,
                     help="destination rows in the CPU-oracle sample (0: 16384 per step of --impl reference, "

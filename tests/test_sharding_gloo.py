@@ -49,6 +49,12 @@ def _worker(rank, world, port, f, cw, result_path):
         full = sharding.gather_columns(torch.from_numpy(local), f, cw)
         want = orc.aggregate("gcn", row_ptr, col, x, f, cw)[0]
         ok = np.array_equal(full.numpy(), want)
+        # the in-place form the GPU ranks use: every rank holds the full-width output, has filled only its own
+        # columns (the others hold a sentinel), and one all-gather completes it
+        mine = torch.full((n, f + 3), -777.0, dtype=torch.float64)          # three padding columns stay untouched
+        mine[:, j0:j1] = torch.from_numpy(local)
+        sharding.gather_slabs_(mine, f, cw)
+        ok = ok and np.array_equal(mine[:, :f].numpy(), want) and bool((mine[:, f:] == -777.0).all())
         ms, units = sharding.reduce_job_timing(10.0 + rank, 100.0 * (rank + 1))
         ok = ok and ms == 10.0 + world - 1 and units == 100.0 * world * (world + 1) / 2
         flag = torch.tensor([1 if ok else 0])
