@@ -586,7 +586,7 @@ def run_ours(args):
             dt = time.perf_counter() - t0
             result["cpu_baseline"] = {"value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
                                       "seconds": dt, "sample": sample_text(w, len(rows)),
-                                      "single_core": oracle_single_core(w, max(len(rows) // 32, 64), [cw])}
+                                      "single_core": oracle_single_core(w, max(len(rows) // 8, 64), [cw])}
         print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()

@@ -43,7 +43,9 @@ typedef enum { GNNFD_I32 = 0, GNNFD_I64 = 1 } gnnfd_itype_t;
 enum {
     GNNFD_CSR_ADD_SELF_LOOPS = 1, /* drop every input loop, then add exactly one (v,v) per vertex */
     GNNFD_CSR_DEDUP = 2,          /* keep the first (lowest edge id) of equal (dst, src) pairs */
-    GNNFD_CSR_SYMMETRIZE = 4      /* add the reverse of every non-loop edge, with edge id e + i */
+    GNNFD_CSR_SYMMETRIZE = 4,     /* add the reverse of every non-loop edge, with edge id e + i */
+    GNNFD_CSR_INPUT_ORDER = 8     /* light build: sort by destination only; the entries of a row keep the order of
+                                     their edge ids instead of ascending source ids (not with DEDUP) */
 };
 
 typedef enum {
@@ -70,6 +72,13 @@ typedef enum {
  * weight deg(src)^-1/2 * deg(dst)^-1/2 per slot, and the launch schedule (rows
  * grouped by degree, rows above GNNFD_HUB_DEGREE cut into segments of
  * GNNFD_HUB_SEGMENT edges).
+ *
+ * GNNFD_CSR_INPUT_ORDER is for graphs that are aggregated once or a few times at a narrow width, where the
+ * conversion would cost more than the aggregation it serves (Section III, the discussion of format-conversion
+ * latency: a conversion can cancel the gain of the format).  The sort then runs over the destination bits only
+ * (half the passes), rows list their sources in edge-id order, and everything else (perm, weights, schedule)
+ * is as above, so every aggregation entry point takes the handle; results differ from the fully ordered
+ * build only in the order of the fp32 additions inside a row.
  */
 #define GNNFD_HUB_DEGREE 2048
 #define GNNFD_HUB_SEGMENT 1024
@@ -184,6 +193,28 @@ int gnnfd_aggregate_gcn_static(const gnnfd_csr_t* csr, const void* d_x, int64_t 
                                void* d_out, int64_t ldo, gnnfd_dtype_t odt, int32_t f, int32_t chunk_width,
                                void* stream);
 
+/* ------------------------------------------------------------------ one-shot aggregation of a COO edge list
+ *
+ * Edge list in, aggregated features out, for a graph that is used once (or at a narrow width, where a full
+ * conversion costs several times the aggregation it serves; Section III of the paper makes that point about
+ * conversion latency, its own method taking the COO edge set as it is).  The call does the light build
+ * (GNNFD_CSR_INPUT_ORDER: half the sort passes; with GNNFD_CSR_DEDUP in `flags` the fully ordered build instead)
+ * and the GCN / SAGE aggregation defined above out of ONE caller buffer, and returns no handle.  Still no
+ * atomics: the stable destination sort fixes the order of every row's additions, so results are bit-identical
+ * from run to run.  d_scratch: gnnfd_oneshot_workspace_bytes(n, e, flags, f) bytes, 256-byte aligned; it holds the
+ * CSR, the sort buffers and the hub-row partial sums (sized for the worst case, because the graph is not known
+ * yet).  Other arguments as for gnnfd_build_csr and gnnfd_aggregate_gcn.  Synchronises the stream once (the build
+ * reads its counters), then enqueues the aggregation. */
+int gnnfd_oneshot_workspace_bytes(int64_t n, int64_t e, uint32_t flags, int32_t f, size_t* scratch_bytes);
+
+int gnnfd_oneshot_gcn(int64_t n, int64_t e, const void* d_src, const void* d_dst, gnnfd_itype_t itype, uint32_t flags,
+                      const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                      int32_t f, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
+
+int gnnfd_oneshot_sage(int64_t n, int64_t e, const void* d_src, const void* d_dst, gnnfd_itype_t itype, uint32_t flags,
+                       const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                       int32_t f, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
+
 /* ------------------------------------------------------------------ GAT
  *
  * The attention aggregator is the third model the paper evaluates (Section II-A lists it with GCN and
@@ -244,18 +275,65 @@ int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float
  *
  * d_x [n, ldx] and d_w_t [f_out, ldw] (the weight matrix transposed: one row per output column) both of
  * type xdt; d_z [n, ldz] of type zdt.  The product runs on the tensor cores with fp32 sums:
- *   xdt = GNNFD_F32 : both operands are read as tf32 (the low 13 mantissa bits of each fp32 value are
- *                     ignored), products are exact, so |z - exact| <= 2^-9 * sum_k |x[v,k] * w_t[j,k]|
+ *   xdt = GNNFD_F32, mode GNNFD_COMBINE_TF32: both operands are read as tf32 (the low 13 mantissa bits of each
+ *                     fp32 value are ignored), products are exact, so |z - exact| <= 2^-9 * sum_k |x[v,k] * w_t[j,k]|
  *                     plus fp32 summation error;
- *   xdt = GNNFD_BF16: operands are used as they are, products are exact in fp32.
+ *   xdt = GNNFD_F32, mode GNNFD_COMBINE_FP32: fp32-faithful.  Each operand is used as a tf32 pair (hi, lo) and
+ *                     the three products that matter are accumulated, so the result meets the library's fp32
+ *                     bar |z - exact| <= 1e-5 * sum_k |x[v,k] * w_t[j,k]| + 1e-6 (the paper's framework runs
+ *                     the Combination in fp32);
+ *   xdt = GNNFD_BF16: operands are used as they are, products are exact in fp32 (mode is ignored).
  * zdt = GNNFD_BF16 rounds the fp32 result to nearest even.
  * d_x and d_w_t must be 16-byte aligned with row pitches that are multiples of 16 bytes
  * (GNNFD_UNSUPPORTED otherwise); d_z has no alignment rule.  d_status (may be NULL): one int32 the caller
  * has set to 0; it becomes 1 if a block gave up waiting for its own copies or matrix instructions (each
- * wait is limited to one second), in which case d_z is incomplete.  The call only enqueues work. */
+ * wait is limited to one second), in which case d_z is incomplete.  The calls only enqueue work.
+ *
+ * gnnfd_combine is the tf32 product alone.  gnnfd_combine_ex adds the mode and, optionally, the GAT scores of
+ * the result as part of the same pass (all four of d_a_src, d_a_dst [heads, dim] and d_s_src, d_s_dst
+ * [n, heads] given, heads * dim == f_out; all four NULL to leave them out): the scores are formed from the
+ * values written to d_z while a thread still holds its output row, so z is not read again.  With more than 256
+ * output columns the columns are processed in tiles, which must then hold whole heads (GNNFD_UNSUPPORTED
+ * otherwise; use gnnfd_gat_scores on the result instead). */
+typedef enum { GNNFD_COMBINE_TF32 = 0, GNNFD_COMBINE_FP32 = 1 } gnnfd_combine_mode_t;
+
 int gnnfd_combine(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t,
                   int64_t ldw, int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int32_t* d_status,
                   void* stream);
+
+int gnnfd_combine_ex(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t,
+                     int64_t ldw, int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int mode,
+                     const float* d_a_src, const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src,
+                     float* d_s_dst, int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------ a whole layer on a built CSR
+ *
+ * Combination, then Aggregation of the transformed features (Section III: the Combination phase is run ahead
+ * of the Aggregation phase, so that Algorithm 1's decomposed aggregation works on the f_out transformed columns
+ * instead of the f_in input columns): out = Aggregate(x * W), with the aggregators defined above.
+ *   gnnfd_layer_gcn / gnnfd_layer_sage : gnnfd_combine_ex, then gnnfd_aggregate_gcn / gnnfd_aggregate_sage.
+ *   gnnfd_layer_gat : gnnfd_combine_ex with the attention scores formed in its epilogue, then the fused GAT
+ *                     aggregation on those scores (no separate scores pass; heads * dim output columns).
+ * x, w_t, mode, d_status as for gnnfd_combine_ex; out, chunk_width as for the aggregation calls (chunk_width
+ * decomposes the f_out transformed columns).  The transformed features z [n, f_out rounded up to 8] are kept in
+ * the scratch buffer in the dtype of x.  d_scratch: gnnfd_layer_workspace_bytes(csr, model, f_out, heads, dim,
+ * xdt) bytes, 256-byte aligned (model 0 = GCN, 1 = SAGE, 2 = GAT; heads and dim are ignored for 0 and 1).
+ * d_out must not alias d_x.  The calls only enqueue work. */
+int gnnfd_layer_workspace_bytes(const gnnfd_csr_t* csr, int model, int32_t f_out, int32_t heads, int32_t dim,
+                                gnnfd_dtype_t xdt, size_t* scratch_bytes);
+
+int gnnfd_layer_gcn(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in,
+                    const void* d_w_t, int64_t ldw, int32_t f_out, int mode, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                    int32_t chunk_width, void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream);
+
+int gnnfd_layer_sage(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in,
+                     const void* d_w_t, int64_t ldw, int32_t f_out, int mode, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                     int32_t chunk_width, void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream);
+
+int gnnfd_layer_gat(const gnnfd_csr_t* csr, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in,
+                    const void* d_w_t, int64_t ldw, int32_t heads, int32_t dim, const float* d_a_src,
+                    const float* d_a_dst, float negative_slope, int mode, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                    int32_t chunk_width, void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream);
 
 /* ------------------------------------------------------------------ diagnostics */
 
@@ -273,6 +351,15 @@ int64_t gnnfd_launch_count(void);
  * distinct kernels seen (may exceed capacity), or a negative status. */
 int gnnfd_kernel_timing_enable(int on);
 int gnnfd_kernel_timing_read(const char** names, double* ms, int64_t* launches, int capacity);
+
+/* Drill of gnnfd_combine's give-up path, for tests.  (The paper has no counterpart.)  It arms the NEXT
+ * gnnfd_combine / gnnfd_combine_ex / gnnfd_layer_* call made by this host thread, and only that one: every
+ * barrier wait of that launch is limited to wait_ns nanoseconds (0 keeps the usual second; at most 10^9) and the
+ * loads of K block skip_k_block (32 fp32 or 64 bf16 columns of x per block; -1: none) are never issued.
+ * Nothing is in flight for the block that was left out, so the waits of the other lanes run out, every thread
+ * block sets *d_status to 1, releases its tensor memory and returns; the device stays usable and d_z is
+ * incomplete. */
+int gnnfd_debug_combine_fault(int64_t wait_ns, int32_t skip_k_block);
 
 #ifdef __cplusplus
 }

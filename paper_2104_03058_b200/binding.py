@@ -15,9 +15,10 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 I32, I64 = 0, 1
-CSR_ADD_SELF_LOOPS, CSR_DEDUP, CSR_SYMMETRIZE = 1, 2, 4
+CSR_ADD_SELF_LOOPS, CSR_DEDUP, CSR_SYMMETRIZE, CSR_INPUT_ORDER = 1, 2, 4, 8
 OK, INVALID_ARG, BAD_INDEX, TOO_LARGE, WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA_ERROR = 0, -1, -2, -3, -4, -5, -6
 STATIC_SCRATCH_EXCEEDED = -7
+COMBINE_TF32, COMBINE_FP32 = 0, 1
 STATIC_SCRATCH_BYTES = 32 << 20
 HUB_DEGREE, HUB_SEGMENT = 2048, 1024
 
@@ -55,6 +56,10 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_aggregate_gcn.argtypes = agg
         L.gnnfd_aggregate_sage.argtypes = agg
         L.gnnfd_aggregate_gcn_static.argtypes = [vp, vp, i64, i32, vp, i64, i32, i32, i32, vp]
+        L.gnnfd_oneshot_workspace_bytes.argtypes = [i64, i64, u32, i32, pp(sz)]
+        one = [i64, i64, vp, vp, i32, u32, vp, i64, i32, vp, i64, i32, i32, i32, vp, sz, vp]
+        L.gnnfd_oneshot_gcn.argtypes = one
+        L.gnnfd_oneshot_sage.argtypes = one
         L.gnnfd_default_chunk_candidates.argtypes = [i32, i32, pp(i32), ctypes.c_int]
         L.gnnfd_tune_chunk_width.argtypes = [vp, ctypes.c_int, vp, i64, i32, vp, i64, i32, i32, pp(i32), ctypes.c_int,
                                              vp, sz, vp, pp(i32), pp(fl)]
@@ -64,6 +69,15 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_edge_softmax_workspace_bytes.argtypes = [vp, i32, pp(sz)]
         L.gnnfd_edge_softmax.argtypes = [vp, vp, vp, i32, fl, vp, vp, sz, vp]
         L.gnnfd_combine.argtypes = [i64, vp, i64, i32, i32, vp, i64, i32, vp, i64, i32, vp, vp]
+        L.gnnfd_combine_ex.argtypes = [i64, vp, i64, i32, i32, vp, i64, i32, vp, i64, i32, ctypes.c_int, vp, vp, i32, i32,
+                                       vp, vp, vp, vp]
+        L.gnnfd_layer_workspace_bytes.argtypes = [vp, ctypes.c_int, i32, i32, i32, i32, pp(sz)]
+        layer = [vp, vp, i64, i32, i32, vp, i64, i32, ctypes.c_int, vp, i64, i32, i32, vp, sz, vp, vp]
+        L.gnnfd_layer_gcn.argtypes = layer
+        L.gnnfd_layer_sage.argtypes = layer
+        L.gnnfd_layer_gat.argtypes = [vp, vp, i64, i32, i32, vp, i64, i32, i32, vp, vp, fl, ctypes.c_int, vp, i64, i32, i32,
+                                      vp, sz, vp, vp]
+        L.gnnfd_debug_combine_fault.argtypes = [i64, i32]
         L.gnnfd_status_string.argtypes = [ctypes.c_int]
         L.gnnfd_status_string.restype = ctypes.c_char_p
         L.gnnfd_last_cuda_error.restype = ctypes.c_int
@@ -284,6 +298,41 @@ def aggregate_sage(csr: Csr, x: torch.Tensor, f: int | None = None, chunk_width:
                       scratch, stream)
 
 
+def oneshot_workspace_bytes(n: int, e: int, flags: int, f: int) -> int:
+    s = ctypes.c_size_t()
+    _check(lib().gnnfd_oneshot_workspace_bytes(n, e, flags, f, ctypes.byref(s)), "gnnfd_oneshot_workspace_bytes")
+    return s.value
+
+
+def oneshot(model: str, n: int, src: torch.Tensor, dst: torch.Tensor, x: torch.Tensor, flags: int = 0, f: int | None = None,
+            chunk_width: int | None = None, out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None):
+    """gnnfd_oneshot_gcn / gnnfd_oneshot_sage: light build + aggregation of a COO edge list in one call."""
+    if not (src.is_cuda and dst.is_cuda) or src.dtype != dst.dtype or src.shape != dst.shape or src.dim() != 1:
+        raise ValueError("src and dst must be 1-D CUDA tensors of the same dtype and length")
+    if src.dtype not in (torch.int32, torch.int64):
+        raise TypeError("edge ids must be int32 or int64")
+    src, dst = src.contiguous(), dst.contiguous()
+    f = x.shape[1] if f is None else f
+    chunk_width = f if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((n, f), dtype=out_dtype or torch.float32, device=x.device)
+    xp, ldx = _matrix(x, f, "x")
+    op, ldo = _matrix(out, f, "out")
+    _same_device(src.device, dst=dst, x=x, out=out)
+    _need_rows(x, n, "x")
+    _need_rows(out, n, "out")
+    _no_overlap(x, out, "x", "out")
+    if scratch is None:
+        scratch = _alloc_bytes(oneshot_workspace_bytes(n, src.numel(), flags, f), x.device, stream)
+    _same_device(src.device, scratch=scratch)
+    fn = {"gcn": lib().gnnfd_oneshot_gcn, "sage": lib().gnnfd_oneshot_sage}[model]
+    _check(fn(n, src.numel(), ctypes.c_void_p(src.data_ptr()), ctypes.c_void_p(dst.data_ptr()),
+              I32 if src.dtype == torch.int32 else I64, flags, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f,
+              chunk_width, ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
+              _stream_ptr(stream)), "gnnfd_oneshot_" + model)
+    return out
+
+
 def default_chunk_candidates(f: int, dtype=torch.float32) -> list:
     buf = (ctypes.c_int32 * 16)()
     k = lib().gnnfd_default_chunk_candidates(f, F32 if dtype == torch.float32 else BF16, buf, 16)
@@ -423,11 +472,22 @@ def edge_softmax(csr: Csr, s_src: torch.Tensor, s_dst: torch.Tensor, negative_sl
     return out
 
 
+def _combine_mode(mode) -> int:
+    if mode in (COMBINE_TF32, "tf32"):
+        return COMBINE_TF32
+    if mode in (COMBINE_FP32, "fp32"):
+        return COMBINE_FP32
+    raise ValueError("mode must be 'tf32' or 'fp32'")
+
+
 def combine(x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, out: torch.Tensor | None = None,
-            out_dtype=None, status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """gnnfd_combine: z = x[:, :f_in] @ w_t[:, :f_in].T on the tensor cores (tf32 operands for float32
-    inputs, bf16 operands for bfloat16 inputs; fp32 sums).  ``status`` is an int32 tensor of one element
-    that the kernel sets to 1 if a block gave up waiting."""
+            out_dtype=None, status: torch.Tensor | None = None, stream=None, mode="tf32", a_src=None, a_dst=None,
+            heads: int = 0, dim: int = 0):
+    """gnnfd_combine_ex: z = x[:, :f_in] @ w_t[:, :f_in].T on the tensor cores with fp32 sums.  float32 inputs
+    are multiplied as tf32 (``mode="tf32"``) or fp32-faithfully as tf32 pairs (``mode="fp32"``); bfloat16 inputs
+    as they are.  ``status`` is an int32 tensor of one element that the kernel sets to 1 if a block gave up
+    waiting.  With ``a_src`` / ``a_dst`` ([heads, dim], heads * dim == f_out) the GAT scores of z are formed in
+    the same pass and the call returns (z, s_src, s_dst) instead of z."""
     f_in = w_t.shape[1] if f_in is None else f_in
     f_out = w_t.shape[0]
     if x.dtype != w_t.dtype:
@@ -442,9 +502,72 @@ def combine(x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, out: to
     _no_overlap(x, out, "x", "out")
     _no_overlap(w_t, out, "w_t", "out")
     sp = ctypes.c_void_p(status.data_ptr()) if status is not None else None
-    _check(lib().gnnfd_combine(x.shape[0], xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, op, ldo, _dtype_code(out), sp,
-                               _stream_ptr(stream)), "gnnfd_combine")
+    scores = a_src is not None or a_dst is not None
+    s_src = s_dst = None
+    asp = adp = ssp = sdp = None
+    if scores:
+        a_src, a_dst = _attention_vectors(a_src, a_dst, heads, dim, x.device, stream)
+        s_src = torch.empty((x.shape[0], heads), dtype=torch.float32, device=x.device)
+        s_dst = torch.empty((x.shape[0], heads), dtype=torch.float32, device=x.device)
+        asp, adp = ctypes.c_void_p(a_src.data_ptr()), ctypes.c_void_p(a_dst.data_ptr())
+        ssp, sdp = ctypes.c_void_p(s_src.data_ptr()), ctypes.c_void_p(s_dst.data_ptr())
+    _check(lib().gnnfd_combine_ex(x.shape[0], xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, op, ldo, _dtype_code(out),
+                                  _combine_mode(mode), asp, adp, heads, dim, ssp, sdp, sp, _stream_ptr(stream)),
+           "gnnfd_combine_ex")
+    return (out, s_src, s_dst) if scores else out
+
+
+def layer_workspace_bytes(csr: Csr, model: str, f_out: int, heads: int = 0, dim: int = 0, dtype=torch.float32) -> int:
+    s = ctypes.c_size_t()
+    _check(lib().gnnfd_layer_workspace_bytes(csr.handle, {"gcn": 0, "sage": 1, "gat": 2}[model], f_out, heads, dim,
+                                             F32 if dtype == torch.float32 else BF16, ctypes.byref(s)),
+           "gnnfd_layer_workspace_bytes")
+    return s.value
+
+
+def layer(csr: Csr, model: str, x: torch.Tensor, w_t: torch.Tensor, f_in: int | None = None, mode="tf32",
+          chunk_width: int | None = None, out: torch.Tensor | None = None, out_dtype=None, a_src=None, a_dst=None,
+          heads: int = 0, dim: int = 0, negative_slope: float = 0.2, scratch=None, status=None, stream=None):
+    """gnnfd_layer_gcn / _sage / _gat: out = Aggregate(x[:, :f_in] @ w_t[:, :f_in].T) on a built CSR; the
+    transformed features stay in the scratch buffer."""
+    f_in = w_t.shape[1] if f_in is None else f_in
+    f_out = w_t.shape[0]
+    if x.dtype != w_t.dtype:
+        raise TypeError("x and w_t must have the same dtype")
+    if model == "gat" and heads * dim != f_out:
+        raise ValueError("heads * dim must equal the number of rows of w_t")
+    chunk_width = f_out if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((csr.n, f_out), dtype=out_dtype or torch.float32, device=x.device)
+    xp, ldx = _matrix(x, f_in, "x")
+    wp, ldw = _matrix(w_t, f_in, "w_t")
+    op, ldo = _matrix(out, f_out, "out")
+    _same_device(csr.device, x=x, w_t=w_t, out=out, status=status)
+    _need_rows(x, csr.n, "x")
+    _need_rows(out, csr.n, "out")
+    _no_overlap(x, out, "x", "out")
+    _no_overlap(w_t, out, "w_t", "out")
+    if scratch is None:
+        scratch = _alloc_bytes(layer_workspace_bytes(csr, model, f_out, heads, dim, x.dtype), x.device, stream)
+    _same_device(csr.device, scratch=scratch)
+    sp = ctypes.c_void_p(status.data_ptr()) if status is not None else None
+    scr, scr_n = ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size()
+    if model == "gat":
+        a_src, a_dst = _attention_vectors(a_src, a_dst, heads, dim, x.device, stream)
+        _check(lib().gnnfd_layer_gat(csr.handle, xp, ldx, _dtype_code(x), f_in, wp, ldw, heads, dim,
+                                     ctypes.c_void_p(a_src.data_ptr()), ctypes.c_void_p(a_dst.data_ptr()), negative_slope,
+                                     _combine_mode(mode), op, ldo, _dtype_code(out), chunk_width, scr, scr_n, sp,
+                                     _stream_ptr(stream)), "gnnfd_layer_gat")
+    else:
+        fn = lib().gnnfd_layer_gcn if model == "gcn" else lib().gnnfd_layer_sage
+        _check(fn(csr.handle, xp, ldx, _dtype_code(x), f_in, wp, ldw, f_out, _combine_mode(mode), op, ldo,
+                  _dtype_code(out), chunk_width, scr, scr_n, sp, _stream_ptr(stream)), "gnnfd_layer_" + model)
     return out
+
+
+def debug_combine_fault(wait_ns: int, skip_k_block: int):
+    """gnnfd_debug_combine_fault: arms the give-up drill for this thread's next transform launch."""
+    _check(lib().gnnfd_debug_combine_fault(wait_ns, skip_k_block), "gnnfd_debug_combine_fault")
 
 
 def launch_count() -> int:

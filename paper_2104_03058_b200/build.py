@@ -13,7 +13,7 @@ INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libgnnfd.so")
 _OBJ_DIR = os.path.join(_PKG, "_build")
 
-SOURCES = ["runtime.cu", "csr_build.cu", "aggregate.cu", "aggregate_static.cu", "gat.cu", "edge_softmax.cu", "tune.cu", "combine.cu"]
+SOURCES = ["runtime.cu", "csr_build.cu", "aggregate.cu", "aggregate_static.cu", "gat.cu", "edge_softmax.cu", "tune.cu", "combine.cu", "layer.cu", "oneshot.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

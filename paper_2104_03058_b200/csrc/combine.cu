@@ -15,6 +15,18 @@
 // i.e. one output row per thread) and store it.  Rows past n and columns past f_in are filled with
 // zeros by the TMA unit, so ragged sizes need no special tiles.
 //
+// fp32-faithful mode (fp32 inputs only): a tf32 operand keeps 10 mantissa bits, which is 50 x coarser than the
+// fp32 arithmetic a framework runs the Combination in.  In this mode every operand value v is used as the pair
+// (hi, lo) with hi = v cut to tf32 (the tensor core does that cut itself when it reads v) and lo = v - hi (exact
+// in fp32, then cut to tf32 by the read), and the product is accumulated as x_lo w_hi + x_hi w_lo + x_hi w_hi:
+// three MMAs per K slice.  The extra warps of the block compute the lo tiles in shared memory (same swizzled
+// layout, element by element) as soon as a stage has landed.  What is dropped is x_lo w_lo (below 2^-20 of the
+// product) and the low bits of lo (below 2^-21).
+//
+// GAT scores from the epilogue: a thread holds a whole row of the output tile in registers, so the two
+// attention scores per head (dot products of the head's columns with a_src / a_dst) are formed there and z
+// is not read again by a separate scores pass.
+//
 // Every wait on a barrier is bounded: when a limit runs out the block records an error in the
 // caller's status word, drains the copies it has in flight (again bounded), frees its tensor memory
 // and returns.
@@ -26,19 +38,32 @@
 namespace gnnfd {
 
 constexpr int kCombineThreads = 128;
+constexpr int kSplitThreads = 256;          // fp32-faithful mode: warps 2..7 compute the lo tiles
 constexpr int kTileM = 128;                 // rows of x per block (the MMA's M)
 constexpr int kTileKBytes = 128;            // bytes per stage row: one 128-byte swizzle span (32 floats or 64 bf16)
 constexpr int kMmaKBytes = 32;              // depth of one MMA: K = 8 for tf32, K = 16 for bf16
 constexpr int kMaxTileN = 256;
 constexpr uint64_t kWaitNs = 1000000000ull; // one second on one barrier before the block gives up
 constexpr int kSmemBudget = 100 * 1024;     // per block, so that two blocks share an SM
+constexpr int kSmemBudgetSplit = 108 * 1024; // fp32-faithful mode (hi and lo tiles per stage): still two blocks per SM
+constexpr int kSmemBudgetMax = 200 * 1024;  // fp32-faithful mode with wide tiles: one block per SM
 constexpr int kMaxStages = 4;
 
 struct CombineArgs {
     void* z;
     int64_t ldz;
     int32_t n, f_in, f_out, tile_n, stages, tmem_cols, z_bf16;
+    int32_t acc_cols, n_main;   // tensor-memory columns per accumulator; accumulators the K blocks rotate over
     int32_t* status;        // set to 1 when a wait ran out (may be null)
+    // GAT scores formed in the epilogue (all null / 0 when not wanted): a_src / a_dst [heads * dim] over the
+    // output columns, s_src / s_dst [n, heads]
+    const float* a_src;
+    const float* a_dst;
+    float* s_src;
+    float* s_dst;
+    int32_t heads, dim;
+    uint64_t wait_ns;       // limit of one barrier wait
+    int32_t skip_k_block;   // fault drill: the producer leaves this K block's loads out (-1: none)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -75,15 +100,20 @@ __device__ __forceinline__ bool mbar_test(uint32_t addr, uint32_t parity)
     return done != 0;
 }
 
-// true once the phase with the given parity has completed; gives up after kWaitNs
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+// true once the phase with the given parity has completed; gives up after limit_ns
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns)
 {
     const uint32_t addr = smem_u32(bar);
     if (mbar_test(addr, parity)) return true;
     const uint64_t t0 = now_ns();
     while (!mbar_test(addr, parity))
-        if (now_ns() - t0 > kWaitNs) return false;
+        if (now_ns() - t0 > limit_ns) return false;
     return true;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int32_t x, int32_t y)
@@ -162,33 +192,71 @@ __device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
 }
 
-template <bool BF16>
-__global__ void __launch_bounds__(kCombineThreads)
+// Adds one output value to the running attention scores of its row; at the last column of a head the two
+// scores are written and the sums start again.  `d` is the column's position inside its head.
+struct ScoreState {
+    float ss, sd;
+    int d, head;
+};
+
+__device__ __forceinline__ void score_step(ScoreState& st, float val, int col, const CombineArgs& a, int row, const float* a_src_s,
+                                           const float* a_dst_s, int col0)
+{
+    st.ss = fmaf(a_src_s[col - col0], val, st.ss);
+    st.sd = fmaf(a_dst_s[col - col0], val, st.sd);
+    if (++st.d == a.dim) {
+        a.s_src[(int64_t)row * a.heads + st.head] = st.ss;
+        a.s_dst[(int64_t)row * a.heads + st.head] = st.sd;
+        st.ss = st.sd = 0.f;
+        st.d = 0;
+        ++st.head;
+    }
+}
+
+// SPLIT: fp32-faithful mode (fp32 operands as tf32 hi + lo pairs, three MMAs per K slice); launched with
+// kSplitThreads threads, of which warps 2.. compute the lo tiles.
+template <bool BF16, bool SPLIT>
+__global__ void __launch_bounds__(SPLIT ? kSplitThreads : kCombineThreads)
 combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CombineArgs a)
 {
+    static_assert(!(BF16 && SPLIT), "bf16 operands are used as they are");
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], split_bar[kMaxStages], accum_bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ float a_src_s[kMaxTileN], a_dst_s[kMaxTileN];
 
     // the dynamic buffer is aligned to 1024 bytes by hand (the swizzle pattern repeats every 1024 bytes)
     unsigned char* tiles = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int kTileK = kTileKBytes / (BF16 ? 2 : 4);      // elements of K per stage
+    constexpr int kSplitWarps = SPLIT ? kSplitThreads / 32 - 2 : 0;
     const uint32_t a_bytes = kTileM * kTileKBytes;
     const uint32_t b_bytes = (uint32_t)a.tile_n * kTileKBytes;
-    const uint32_t stage_bytes = a_bytes + b_bytes;
+    const uint32_t stage_bytes = a_bytes + b_bytes;            // what the TMA unit delivers per stage
+    const uint32_t stage_pitch = SPLIT ? 2 * stage_bytes : stage_bytes;   // the lo tiles follow the loaded ones
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row0 = blockIdx.x * kTileM;
     const int col0 = blockIdx.y * a.tile_n;
     const int k_blocks = (a.f_in + kTileK - 1) / kTileK;
+    const bool want_scores = a.s_src != nullptr;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < a.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < a.stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+            mbar_init(&split_bar[s], SPLIT ? kSplitWarps : 1);
+        }
         mbar_init(&accum_bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (want_scores)
+        for (int c = threadIdx.x; c < a.tile_n; c += blockDim.x) {
+            const bool in = col0 + c < a.f_out;
+            a_src_s[c] = in ? a.a_src[col0 + c] : 0.f;
+            a_dst_s[c] = in ? a.a_dst[col0 + c] : 0.f;
+        }
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"((uint32_t)a.tmem_cols)
@@ -200,67 +268,124 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
 
+    int issued = 0;            // K blocks the producer lane has gone through (thread 0 only)
     if (warp == 0 && lane == 0) {
         // producer: fills stage kb % stages once the MMAs that read its previous contents have finished
-        int issued = 0;
         bool ok = true;
         for (int kb = 0; kb < k_blocks && ok; ++kb) {
             const int s = kb % a.stages;
-            if (kb >= a.stages) ok = mbar_wait(&empty_bar[s], ((kb / a.stages) - 1) & 1);
+            if (kb >= a.stages) ok = mbar_wait(&empty_bar[s], ((kb / a.stages) - 1) & 1, a.wait_ns);
             if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
-            unsigned char* stage = tiles + (size_t)s * stage_bytes;
+            issued = kb + 1;
+            if (kb == a.skip_k_block) continue;        // fault drill: nothing is issued for this block, so nothing of it is in flight
+            unsigned char* stage = tiles + (size_t)s * stage_pitch;
             mbar_expect_tx(&full_bar[s], stage_bytes);
             tma_load_2d(stage, &map_x, &full_bar[s], kb * kTileK, row0);
             tma_load_2d(stage + a_bytes, &map_w, &full_bar[s], kb * kTileK, col0);
-            issued = kb + 1;
         }
-        if (!ok) {
-            *(volatile int*)&abort_flag = 1;
-            // the copies already issued must land before the block's shared memory is given back
-            const int first = issued > a.stages ? issued - a.stages : 0;
-            for (int kb = first; kb < issued; ++kb) mbar_wait(&full_bar[kb % a.stages], (kb / a.stages) & 1);
-        }
+        if (!ok) *(volatile int*)&abort_flag = 1;
     } else if (warp == 1 && lane == 0) {
         // MMA issuer
         const uint32_t idesc = instr_desc<BF16>(a.tile_n);
         bool ok = true;
         for (int kb = 0; kb < k_blocks && ok; ++kb) {
             const int s = kb % a.stages;
-            ok = mbar_wait(&full_bar[s], (kb / a.stages) & 1);
+            ok = mbar_wait(SPLIT ? &split_bar[s] : &full_bar[s], (kb / a.stages) & 1, a.wait_ns);
             if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+            const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_pitch);
             const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
             for (int k = 0; k < kTileKBytes / kMmaKBytes; ++k) {
                 // inside the 128-byte swizzle span the next K slice starts 32 bytes further on
                 const uint64_t da = operand_desc(a_addr + k * kMmaKBytes);
                 const uint64_t db = operand_desc(b_addr + k * kMmaKBytes);
-                mma<BF16>(tmem_base, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                // K block kb adds into accumulator kb % n_main: every addition into an accumulator cuts the sum's
+                // low bits, so spreading the additions keeps the chain (and its one-sided drift on same-sign data) short
+                const uint32_t acc = tmem_base + (uint32_t)((kb % a.n_main) * a.acc_cols);
+                const uint32_t carry = (kb >= a.n_main || k > 0) ? 1u : 0u;
+                if constexpr (SPLIT) {
+                    // the two small products go to an accumulator of their own (the last one), where they lose nothing
+                    // against the large sum; the epilogue adds it once
+                    const uint32_t acc_lo = tmem_base + (uint32_t)(a.n_main * a.acc_cols);
+                    const uint64_t da_lo = operand_desc(a_addr + stage_bytes + k * kMmaKBytes);
+                    const uint64_t db_lo = operand_desc(b_addr + stage_bytes + k * kMmaKBytes);
+                    mma<BF16>(acc_lo, da_lo, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    mma<BF16>(acc_lo, da, db_lo, idesc, 1u);
+                    mma<BF16>(acc, da, db, idesc, carry);
+                } else {
+                    mma<BF16>(acc, da, db, idesc, carry);
+                }
             }
             mma_commit(&empty_bar[s]);
         }
         if (ok) mma_commit(&accum_bar);
         else *(volatile int*)&abort_flag = 1;
+    } else if (SPLIT && warp >= 2) {
+        // lo tiles: element by element over the stage (the swizzle only permutes 16-byte pieces, so the lo tile
+        // has the layout of the loaded one), then visible to the tensor core's reads, then one arrival per warp
+        const int t = threadIdx.x - 64;
+        const int n_vec = (int)(stage_bytes / 16);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % a.stages;
+            ok = mbar_wait(&full_bar[s], (kb / a.stages) & 1, a.wait_ns);
+            ok = __all_sync(0xffffffffu, ok && !*(volatile int*)&abort_flag);
+            if (!ok) break;
+            const float4* hi = reinterpret_cast<const float4*>(tiles + (size_t)s * stage_pitch);
+            float4* lo = reinterpret_cast<float4*>(tiles + (size_t)s * stage_pitch + stage_bytes);
+#pragma unroll 4
+            for (int i = t; i < n_vec; i += kSplitWarps * 32) {
+                const float4 v = hi[i];
+                float4 r;
+                r.x = v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+                r.y = v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+                r.z = v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+                r.w = v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+                lo[i] = r;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&split_bar[s]);
+        }
+        if (!ok && lane == 0) *(volatile int*)&abort_flag = 1;
     }
     __syncwarp();
 
-    // epilogue: thread t of warp w holds row 32 w + t of the tile
-    bool ok = mbar_wait(&accum_bar, 0) && !*(volatile int*)&abort_flag;
-    // on an abort the accumulator barrier never completes: all lanes of all warps agree through the flag
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    // epilogue (warps 0 - 3): thread t of warp w holds row 32 w + t of the tile
+    bool ok = true;
+    if (warp < 4) {
+        ok = mbar_wait(&accum_bar, 0, a.wait_ns) && !*(volatile int*)&abort_flag;
+        // on an abort the accumulator barrier never completes: all lanes of all warps agree through the flag
+        ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok && warp < 4) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int row = row0 + warp * 32 + lane;
         const int col_end = min(a.f_out, col0 + a.tile_n);
         const int zsize = a.z_bf16 ? 2 : 4;
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(a.z) | (uintptr_t)(a.ldz * zsize)) & 15u) == 0;
+        ScoreState st{0.f, 0.f, 0, 0};
+        if (want_scores) { st.d = col0 % a.dim; st.head = col0 / a.dim; }     // tiles start on head boundaries (host check)
         for (int c = 0; c < a.tile_n; c += 32) {
             uint32_t r[32];
-            tmem_load_32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+            const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c;
+            tmem_load_32(lane_base, r);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            // the other accumulators that received K blocks, then (fp32-faithful mode) the small products
+            const int used = k_blocks < a.n_main ? k_blocks : a.n_main;
+            for (int j = 1; j < used + (SPLIT ? 1 : 0); ++j) {
+                uint32_t t[32];
+                tmem_load_32(lane_base + (uint32_t)((j < used ? j : a.n_main) * a.acc_cols), t);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(t[i]));
+            }
             if (row >= a.n) continue;
             if (a.z_bf16) {
+                // the stored value is the fp32 sum rounded to bf16; scores are formed from what is stored
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__bfloat162float(__float2bfloat16_rn(__uint_as_float(r[j]))));
                 __nv_bfloat16* zrow = static_cast<__nv_bfloat16*>(a.z) + (int64_t)row * a.ldz + col0 + c;
 #pragma unroll
                 for (int j = 0; j < 32; j += 8) {
@@ -269,10 +394,7 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
                         uint4 v;
                         uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * i]), __uint_as_float(r[j + 2 * i + 1]));
-                            pv[i] = *reinterpret_cast<const uint32_t*>(&h);
-                        }
+                        for (int i = 0; i < 4; ++i) pv[i] = (r[j + 2 * i] >> 16) | (r[j + 2 * i + 1] & 0xffff0000u);
                         __stcs(reinterpret_cast<uint4*>(zrow + j), v);
                     } else {
 #pragma unroll
@@ -296,9 +418,20 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
                     }
                 }
             }
+            if (want_scores) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + c + j < col_end) score_step(st, __uint_as_float(r[j]), col0 + c + j, a, row, a_src_s, a_dst_s, col0);
+            }
         }
-    } else if (threadIdx.x == 0 && a.status) {
-        atomicExch(a.status, 1);
+    } else if (threadIdx.x == 0) {
+        if (a.status) atomicExch(a.status, 1);
+        // This thread is the producer lane.  The copies of the last `stages` K blocks it issued may still be in
+        // flight; they must land before the block's shared memory is given back, so it waits for each of them
+        // once more (bounded).  A block left out by the fault drill has nothing in flight.
+        const int first = issued > a.stages ? issued - a.stages : 0;
+        for (int kb = first; kb < issued; ++kb)
+            if (kb != a.skip_k_block) mbar_wait(&full_bar[kb % a.stages], (kb / a.stages) & 1, a.wait_ns);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -343,50 +476,113 @@ static bool make_map(CUtensorMap* map, const void* base, bool bf16, int64_t rows
 
 }  // namespace gnnfd
 
-extern "C" int gnnfd_combine(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t,
-                             int64_t ldw, int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int32_t* d_status,
-                             void* stream)
+namespace gnnfd {
+
+// One-shot settings of the fault drill (see gnnfd_debug_combine_fault): consumed by the next launch on this thread.
+static thread_local uint64_t t_drill_wait_ns = 0;
+static thread_local int32_t t_drill_skip = -1;
+
+int combine_impl(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t, int64_t ldw,
+                 int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int mode, const float* d_a_src,
+                 const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst, int32_t* d_status,
+                 cudaStream_t s)
 {
-    using namespace gnnfd;
     if (n <= 0 || !d_x || !d_w_t || !d_z || f_in <= 0 || f_out <= 0 || ldx < f_in || ldw < f_in || ldz < f_out)
         return GNNFD_INVALID_ARG;
     if ((xdt != GNNFD_F32 && xdt != GNNFD_BF16) || (zdt != GNNFD_F32 && zdt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
+    if (mode != GNNFD_COMBINE_TF32 && mode != GNNFD_COMBINE_FP32) return GNNFD_INVALID_ARG;
     if (n > 0x7fffffffll - kTileM) return GNNFD_TOO_LARGE;
     const bool bf16 = xdt == GNNFD_BF16;
+    const bool split = !bf16 && mode == GNNFD_COMBINE_FP32;     // bf16 products are exact already
     const int esize = bf16 ? 2 : 4;
     // the TMA unit wants 16-byte aligned bases and row pitches
     if (((uintptr_t)d_x | (uintptr_t)d_w_t) % 16 != 0 || (ldx * esize) % 16 != 0 || (ldw * esize) % 16 != 0)
         return GNNFD_UNSUPPORTED;
+    const bool scores = d_s_src || d_s_dst || d_a_src || d_a_dst;
+    if (scores && (!d_s_src || !d_s_dst || !d_a_src || !d_a_dst || heads <= 0 || dim <= 0 || (int64_t)heads * dim != f_out))
+        return GNNFD_INVALID_ARG;
 
     CombineArgs a;
     a.z = d_z; a.ldz = ldz; a.n = (int32_t)n; a.f_in = f_in; a.f_out = f_out; a.status = d_status;
     a.z_bf16 = zdt == GNNFD_BF16;
+    a.a_src = scores ? d_a_src : nullptr; a.a_dst = scores ? d_a_dst : nullptr;
+    a.s_src = scores ? d_s_src : nullptr; a.s_dst = scores ? d_s_dst : nullptr;
+    a.heads = heads; a.dim = dim;
+    a.wait_ns = t_drill_wait_ns ? t_drill_wait_ns : kWaitNs;
+    a.skip_k_block = t_drill_skip;
+    t_drill_wait_ns = 0;
+    t_drill_skip = -1;
     // output columns per block: all of them up to 256, rounded up to the MMA's N granularity of 16
     const int n_col_tiles = (f_out + kMaxTileN - 1) / kMaxTileN;
     const int per_tile = (f_out + n_col_tiles - 1) / n_col_tiles;
     a.tile_n = (per_tile + 15) / 16 * 16;
-    a.tmem_cols = 32;
-    while (a.tmem_cols < a.tile_n) a.tmem_cols <<= 1;
-    const int stage_bytes = (kTileM + a.tile_n) * kTileKBytes;
-    a.stages = kSmemBudget / stage_bytes;
+    // a head's scores are formed by one thread: with several column tiles every tile must hold whole heads
+    if (scores && n_col_tiles > 1 && a.tile_n % dim != 0) return GNNFD_UNSUPPORTED;
+    a.acc_cols = 32;
+    while (a.acc_cols < a.tile_n) a.acc_cols <<= 1;
+    const int stage_bytes = (kTileM + a.tile_n) * kTileKBytes * (split ? 2 : 1);
+    int budget = split ? kSmemBudgetSplit : kSmemBudget;
+    bool two_per_sm = true;
+    if (budget / stage_bytes < 2) { budget = kSmemBudgetMax; two_per_sm = false; }      // wide tiles: one block per SM
+    // tensor memory: 512 columns per SM, shared by the blocks resident there; all of a block's share becomes accumulators
+    a.tmem_cols = two_per_sm ? 256 : 512;
+    const int n_acc = a.tmem_cols / a.acc_cols;
+    a.n_main = split ? n_acc - 1 : n_acc;
+    if (a.n_main < 1) return GNNFD_UNSUPPORTED;
+    a.stages = budget / stage_bytes;
     if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return GNNFD_UNSUPPORTED;
-    const size_t smem = (size_t)a.stages * stage_bytes + 1024;
+    size_t smem = (size_t)a.stages * stage_bytes + 1024;
+    // each block takes half of the SM's tensor memory, so no more than two may share an SM (a third would sit in
+    // its allocation until one of them left): ask for more than a third of the SM's shared memory
+    if (smem < 80 * 1024) smem = 80 * 1024;
 
     CUtensorMap map_x, map_w;
     if (!make_map(&map_x, d_x, bf16, n, f_in, ldx, kTileM) || !make_map(&map_w, d_w_t, bf16, f_out, f_in, ldw, a.tile_n)) {
         set_cuda_error(cudaErrorInvalidValue);
         return GNNFD_CUDA_ERROR;
     }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     const dim3 grid((unsigned)((n + kTileM - 1) / kTileM), (unsigned)((f_out + a.tile_n - 1) / a.tile_n));
     if (bf16) {
-        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        GNNFD_LAUNCH("combine_bf16", s, combine_mma<true>, grid, kCombineThreads, smem, map_x, map_w, a);
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_bf16", s, (combine_mma<true, false>), grid, kCombineThreads, smem, map_x, map_w, a);
+    } else if (split) {
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_fp32_3xtf32", s, (combine_mma<false, true>), grid, kSplitThreads, smem, map_x, map_w, a);
     } else {
-        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        GNNFD_LAUNCH("combine_tf32", s, combine_mma<false>, grid, kCombineThreads, smem, map_x, map_w, a);
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_tf32", s, (combine_mma<false, false>), grid, kCombineThreads, smem, map_x, map_w, a);
     }
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
 }
+
+}  // namespace gnnfd
+
+extern "C" {
+
+int gnnfd_combine(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t, int64_t ldw,
+                  int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int32_t* d_status, void* stream)
+{
+    return gnnfd::combine_impl(n, d_x, ldx, xdt, f_in, d_w_t, ldw, f_out, d_z, ldz, zdt, GNNFD_COMBINE_TF32, nullptr, nullptr,
+                               0, 0, nullptr, nullptr, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int gnnfd_combine_ex(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t, int64_t ldw,
+                     int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int mode, const float* d_a_src,
+                     const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst, int32_t* d_status,
+                     void* stream)
+{
+    return gnnfd::combine_impl(n, d_x, ldx, xdt, f_in, d_w_t, ldw, f_out, d_z, ldz, zdt, mode, d_a_src, d_a_dst, heads, dim,
+                               d_s_src, d_s_dst, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int gnnfd_debug_combine_fault(int64_t wait_ns, int32_t skip_k_block)
+{
+    if (wait_ns < 0 || wait_ns > 1000000000ll) return GNNFD_INVALID_ARG;
+    gnnfd::t_drill_wait_ns = (uint64_t)wait_ns;
+    gnnfd::t_drill_skip = skip_k_block;
+    return GNNFD_OK;
+}
+
+}  // extern "C"

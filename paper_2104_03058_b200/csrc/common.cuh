@@ -80,6 +80,21 @@ struct Carver {
 size_t scan_temp_ints(size_t count);
 int exclusive_scan_i32(const int32_t* d_in, int32_t* d_out, size_t count, int32_t* d_temp, cudaStream_t s);
 
+// ---- pieces of one translation unit that the layer entry points (layer.cu) put together
+
+int64_t segment_capacity(int64_t n, int64_t e, uint32_t flags);      // csr_build.cu; -1 for sizes the build rejects
+
+int combine_impl(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int32_t f_in, const void* d_w_t, int64_t ldw,
+                 int32_t f_out, void* d_z, int64_t ldz, gnnfd_dtype_t zdt, int mode, const float* d_a_src,
+                 const float* d_a_dst, int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst, int32_t* d_status,
+                 cudaStream_t s);
+int gat_aggregate_impl(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
+                       const float* d_a_dst, int32_t heads, int32_t dim, float negative_slope, void* d_out, int64_t ldo,
+                       gnnfd_dtype_t odt, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, bool scores_ready,
+                       cudaStream_t s);
+int gat_scratch_scores(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, void* d_scratch, size_t scratch_bytes,
+                       float** s_src, float** s_dst);
+
 }  // namespace gnnfd
 
 #define GNNFD_LAUNCH(name, stream, kernel, grid, block, smem, ...)                   \

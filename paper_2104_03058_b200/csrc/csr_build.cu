@@ -532,13 +532,17 @@ struct BuildLayout {
     int64_t hub_cap;       // upper bound on hub rows
     int64_t seg_cap;       // upper bound on hub segments
     int src_bits, key_bits, passes, digit_bits;
+    int first_bit;         // lowest key bit the sort looks at (0; src_bits when rows keep their input order)
     int val_bits;          // > 0: keys and values share one 64-bit word (key << val_bits | value + 1)
 };
 
 static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
 {
     if (n <= 0 || e < 0) return GNNFD_INVALID_ARG;
-    if (flags & ~(uint32_t)(GNNFD_CSR_ADD_SELF_LOOPS | GNNFD_CSR_DEDUP | GNNFD_CSR_SYMMETRIZE)) return GNNFD_INVALID_ARG;
+    if (flags & ~(uint32_t)(GNNFD_CSR_ADD_SELF_LOOPS | GNNFD_CSR_DEDUP | GNNFD_CSR_SYMMETRIZE | GNNFD_CSR_INPUT_ORDER))
+        return GNNFD_INVALID_ARG;
+    // duplicates are found as neighbours of the (dst, src) order, which the input-order build does not establish
+    if ((flags & GNNFD_CSR_INPUT_ORDER) && (flags & GNNFD_CSR_DEDUP)) return GNNFD_INVALID_ARG;
     const int64_t limit = (int64_t(1) << 31) - 1;
     if (n > limit || e > limit) return GNNFD_TOO_LARGE;
     int64_t m = e;
@@ -557,12 +561,23 @@ static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
     while ((int64_t(1) << dst_bits) < n + 1) ++dst_bits;      // destination n marks dropped candidates
     L->src_bits = bits;
     L->key_bits = bits + dst_bits;
-    L->passes = (L->key_bits + kMaxDigitBits - 1) / kMaxDigitBits;
-    L->digit_bits = (L->key_bits + L->passes - 1) / L->passes;
+    // Rows in input order: the stable sort looks at the destination bits only, so entries of a row stay in the
+    // order of their candidate numbers (input edges, then reverses, then the added loop).
+    L->first_bit = (flags & GNNFD_CSR_INPUT_ORDER) ? bits : 0;
+    const int sort_bits = L->key_bits - L->first_bit;
+    L->passes = (sort_bits + kMaxDigitBits - 1) / kMaxDigitBits;
+    L->digit_bits = (sort_bits + L->passes - 1) / L->passes;
     int vb = 1;
     while ((int64_t(1) << vb) < m + 2) ++vb;                  // values -1 .. m-1 stored as 0 .. m
     L->val_bits = L->key_bits + vb <= 64 ? vb : 0;
     return GNNFD_OK;
+}
+
+// upper bound on the hub segments of any graph with these sizes (what the persistent buffer reserves)
+int64_t segment_capacity(int64_t n, int64_t e, uint32_t flags)
+{
+    BuildLayout L;
+    return make_layout(n, e, flags, &L) == GNNFD_OK ? L.seg_cap : -1;
 }
 
 struct PersistentPtrs {
@@ -695,7 +710,7 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
                          L.src_bits, vb, keys, key_vals, P.counts);
         const int mask = (1 << L.digit_bits) - 1;
         for (int pass = 0; pass < L.passes; ++pass) {
-            const int shift = pass * L.digit_bits + vb;
+            const int shift = L.first_bit + pass * L.digit_bits + vb;
             GNNFD_LAUNCH("radix_histogram", s, radix_histogram, (unsigned)L.n_tiles, kThreads, 0, keys, m, shift, mask,
                          L.n_tiles, S.hist);
             rc = exclusive_scan_i32(S.hist, S.hist, (size_t)kRadix * (size_t)L.n_tiles, S.scan_temp, s);

@@ -437,38 +437,15 @@ static int launch_scores(int64_t n, const void* d_z, int64_t ldz, gnnfd_dtype_t 
     return GNNFD_OK;
 }
 
-}  // namespace gnnfd
-
-extern "C" {
-
-int gnnfd_gat_scores(int64_t n, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src, const float* d_a_dst,
-                     int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst, void* stream)
+// scores_ready: the two score arrays at the head of the scratch buffer (see gat_scratch_scores) already hold the
+// scores of d_z (the dense transform's epilogue wrote them), so the scores pass is left out.
+int gat_aggregate_impl(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
+                       const float* d_a_dst, int32_t heads, int32_t dim, float negative_slope, void* d_out, int64_t ldo,
+                       gnnfd_dtype_t odt, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, bool scores_ready,
+                       cudaStream_t s)
 {
-    if (n <= 0 || !d_z || !d_a_src || !d_a_dst || !d_s_src || !d_s_dst || heads <= 0 || dim <= 0 ||
-        ldz < (int64_t)heads * dim)
-        return GNNFD_INVALID_ARG;
-    if (zdt != GNNFD_F32 && zdt != GNNFD_BF16) return GNNFD_UNSUPPORTED;
-    if (n * heads > 0x7fffffffll * gnnfd::kBlock) return GNNFD_TOO_LARGE;
-    return gnnfd::launch_scores(n, d_z, ldz, zdt, d_a_src, d_a_dst, heads, dim, d_s_src, d_s_dst,
-                                static_cast<cudaStream_t>(stream));
-}
-
-int gnnfd_gat_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, size_t* scratch_bytes)
-{
-    if (!csr || heads <= 0 || dim <= 0 || !scratch_bytes) return GNNFD_INVALID_ARG;
-    gnnfd::Carver c(nullptr, ~size_t(0));
-    gnnfd::GatScratch g;
-    gnnfd::carve_gat(c, csr, heads, dim, &g);
-    *scratch_bytes = c.off;
-    return GNNFD_OK;
-}
-
-int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
-                        const float* d_a_dst, int32_t heads, int32_t dim, float negative_slope, void* d_out, int64_t ldo,
-                        gnnfd_dtype_t odt, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream)
-{
-    using namespace gnnfd;
-    if (!csr || !d_z || !d_a_src || !d_a_dst || !d_out || heads <= 0 || dim <= 0 || chunk_width <= 0) return GNNFD_INVALID_ARG;
+    if (!csr || !d_z || !d_out || heads <= 0 || dim <= 0 || chunk_width <= 0) return GNNFD_INVALID_ARG;
+    if (!scores_ready && (!d_a_src || !d_a_dst)) return GNNFD_INVALID_ARG;
     const int64_t f64 = (int64_t)heads * dim;
     if (f64 > 0x7fffffffll || ldz < f64 || ldo < f64 || ldz > 0x7fffffffll) return GNNFD_INVALID_ARG;
     if ((zdt != GNNFD_F32 && zdt != GNNFD_BF16) || (odt != GNNFD_F32 && odt != GNNFD_BF16)) return GNNFD_UNSUPPORTED;
@@ -478,10 +455,10 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     GatScratch g;
     carve_gat(c, csr, heads, dim, &g);
     if (!c.ok) return GNNFD_WORKSPACE_TOO_SMALL;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-
-    int rc = launch_scores(csr->n, d_z, ldz, zdt, d_a_src, d_a_dst, heads, dim, g.s_src, g.s_dst, s);
-    if (rc) return rc;
+    if (!scores_ready) {
+        int rc = launch_scores(csr->n, d_z, ldz, zdt, d_a_src, d_a_dst, heads, dim, g.s_src, g.s_dst, s);
+        if (rc) return rc;
+    }
 
     const int cw = chunk_width < f ? chunk_width : f;
     const int n_chunks = (f + cw - 1) / cw;
@@ -529,6 +506,54 @@ int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gn
     }
     GNNFD_CUDA_CHECK(cudaGetLastError());
     return GNNFD_OK;
+}
+
+// where gnnfd_aggregate_gat keeps the two [n, heads] score arrays inside its scratch buffer
+int gat_scratch_scores(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, void* d_scratch, size_t scratch_bytes,
+                       float** s_src, float** s_dst)
+{
+    if (!csr || heads <= 0 || dim <= 0 || !d_scratch || ((uintptr_t)d_scratch & 255u)) return GNNFD_INVALID_ARG;
+    Carver c(d_scratch, scratch_bytes);
+    GatScratch g;
+    carve_gat(c, csr, heads, dim, &g);
+    if (!c.ok) return GNNFD_WORKSPACE_TOO_SMALL;
+    *s_src = g.s_src;
+    *s_dst = g.s_dst;
+    return GNNFD_OK;
+}
+
+}  // namespace gnnfd
+
+extern "C" {
+
+int gnnfd_gat_scores(int64_t n, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src, const float* d_a_dst,
+                     int32_t heads, int32_t dim, float* d_s_src, float* d_s_dst, void* stream)
+{
+    if (n <= 0 || !d_z || !d_a_src || !d_a_dst || !d_s_src || !d_s_dst || heads <= 0 || dim <= 0 ||
+        ldz < (int64_t)heads * dim)
+        return GNNFD_INVALID_ARG;
+    if (zdt != GNNFD_F32 && zdt != GNNFD_BF16) return GNNFD_UNSUPPORTED;
+    if (n * heads > 0x7fffffffll * gnnfd::kBlock) return GNNFD_TOO_LARGE;
+    return gnnfd::launch_scores(n, d_z, ldz, zdt, d_a_src, d_a_dst, heads, dim, d_s_src, d_s_dst,
+                                static_cast<cudaStream_t>(stream));
+}
+
+int gnnfd_gat_workspace_bytes(const gnnfd_csr_t* csr, int32_t heads, int32_t dim, size_t* scratch_bytes)
+{
+    if (!csr || heads <= 0 || dim <= 0 || !scratch_bytes) return GNNFD_INVALID_ARG;
+    gnnfd::Carver c(nullptr, ~size_t(0));
+    gnnfd::GatScratch g;
+    gnnfd::carve_gat(c, csr, heads, dim, &g);
+    *scratch_bytes = c.off;
+    return GNNFD_OK;
+}
+
+int gnnfd_aggregate_gat(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src,
+                        const float* d_a_dst, int32_t heads, int32_t dim, float negative_slope, void* d_out, int64_t ldo,
+                        gnnfd_dtype_t odt, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream)
+{
+    return gnnfd::gat_aggregate_impl(csr, d_z, ldz, zdt, d_a_src, d_a_dst, heads, dim, negative_slope, d_out, ldo, odt,
+                                     chunk_width, d_scratch, scratch_bytes, false, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
