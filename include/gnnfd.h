@@ -70,8 +70,8 @@ typedef enum {
  * reverse of edge i; -1 for an added self-loop), the degree normalisers
  * deg^-1/2 and 1/deg (0 for empty rows, deg = entries in the row), the GCN edge
  * weight deg(src)^-1/2 * deg(dst)^-1/2 per slot, and the launch schedule (rows
- * grouped by degree, rows above GNNFD_HUB_DEGREE cut into segments of
- * GNNFD_HUB_SEGMENT edges).
+ * grouped by degree, rows above GNNFD_HUB_DEGREE cut into segments of at most
+ * GNNFD_HUB_SEGMENT edges; see gnnfd_csr_schedule).
  *
  * GNNFD_CSR_INPUT_ORDER is for graphs that are aggregated once or a few times at a narrow width, where the
  * conversion would cost more than the aggregation it serves (Section III, the discussion of format-conversion
@@ -82,6 +82,7 @@ typedef enum {
  */
 #define GNNFD_HUB_DEGREE 2048
 #define GNNFD_HUB_SEGMENT 1024
+#define GNNFD_HUB_RANGE_ROWS 65536
 
 /* Sizes (bytes) of the two device buffers gnnfd_build_csr needs for n vertices and e input edges.
  * persistent: must stay alive and untouched while the handle is in use.
@@ -110,11 +111,16 @@ int gnnfd_csr_info(const gnnfd_csr_t* csr, int64_t* n, int64_t* nnz, const int32
  * hub rows.  d_row_order[n]: row ids sorted by degree class, ascending id inside a class; a class is
  * the exact degree up to 8, then a quarter octave of (degree - 1) up to GNNFD_HUB_DEGREE, then one
  * class for all hub rows, so every bin is a contiguous range and neighbouring rows have near-equal
- * lengths.  Hub segments: d_seg_row[n_segments], d_seg_begin[n_segments] (first CSR slot of the
- * segment); d_hub_seg_ptr[n_hub+1] indexes the segments of the i-th hub row (i-th row of the last bin). */
+ * lengths.  Hub rows are cut at the boundaries of source ranges of GNNFD_HUB_RANGE_ROWS vertex ids (doubled
+ * until at most 64 ranges cover the graph; one range for a GNNFD_CSR_INPUT_ORDER build) and then into segments of
+ * at most GNNFD_HUB_SEGMENT entries.  The segment arrays are in launch order, which goes range by range over all
+ * hub rows, so that the hub rows in flight gather from one band of source rows: d_seg_row[n_segments],
+ * d_seg_begin / d_seg_end (CSR slots [begin, end) of the segment), d_seg_slot (the segment's number when a row's
+ * segments are counted in ascending source order, row after row: partial results are stored by slot).
+ * d_hub_seg_ptr[n_hub+1]: the slots of the i-th hub row (i-th row of the last bin) are [ptr[i], ptr[i+1]). */
 int gnnfd_csr_schedule(const gnnfd_csr_t* csr, int64_t bin_count[5], const int32_t** d_row_order,
                        int64_t* n_segments, const int32_t** d_seg_row, const int32_t** d_seg_begin,
-                       const int32_t** d_hub_seg_ptr);
+                       const int32_t** d_seg_end, const int32_t** d_seg_slot, const int32_t** d_hub_seg_ptr);
 
 /* Frees the host-side handle only. */
 void gnnfd_csr_destroy(gnnfd_csr_t* csr);

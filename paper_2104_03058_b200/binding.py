@@ -20,7 +20,7 @@ OK, INVALID_ARG, BAD_INDEX, TOO_LARGE, WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA_ER
 STATIC_SCRATCH_EXCEEDED = -7
 COMBINE_TF32, COMBINE_FP32 = 0, 1
 STATIC_SCRATCH_BYTES = 32 << 20
-HUB_DEGREE, HUB_SEGMENT = 2048, 1024
+HUB_DEGREE, HUB_SEGMENT, HUB_RANGE_ROWS = 2048, 1024, 65536
 
 _lib = None
 
@@ -48,7 +48,7 @@ def lib() -> ctypes.CDLL:
         L.gnnfd_csr_workspace_bytes.argtypes = [i64, i64, u32, pp(sz), pp(sz)]
         L.gnnfd_build_csr.argtypes = [i64, i64, vp, vp, i32, u32, vp, sz, vp, sz, vp, pp(vp)]
         L.gnnfd_csr_info.argtypes = [vp, pp(i64), pp(i64), pp(vp), pp(vp), pp(vp), pp(vp), pp(vp), pp(vp), pp(i32)]
-        L.gnnfd_csr_schedule.argtypes = [vp, pp(i64 * 5), pp(vp), pp(i64), pp(vp), pp(vp), pp(vp)]
+        L.gnnfd_csr_schedule.argtypes = [vp, pp(i64 * 5), pp(vp), pp(i64), pp(vp), pp(vp), pp(vp), pp(vp), pp(vp)]
         L.gnnfd_csr_destroy.argtypes = [vp]
         L.gnnfd_csr_destroy.restype = None
         L.gnnfd_aggregate_workspace_bytes.argtypes = [vp, i32, pp(sz)]
@@ -188,13 +188,15 @@ class Csr:
                               [p.value for p in ptrs]))
         bins = (ctypes.c_int64 * 5)()
         nseg = ctypes.c_int64()
-        sp = [ctypes.c_void_p() for _ in range(4)]
+        sp = [ctypes.c_void_p() for _ in range(6)]
         _check(lib().gnnfd_csr_schedule(self._h, ctypes.byref(bins), ctypes.byref(sp[0]), ctypes.byref(nseg),
-                                        ctypes.byref(sp[1]), ctypes.byref(sp[2]), ctypes.byref(sp[3])),
+                                        ctypes.byref(sp[1]), ctypes.byref(sp[2]), ctypes.byref(sp[3]), ctypes.byref(sp[4]),
+                                        ctypes.byref(sp[5])),
                "gnnfd_csr_schedule")
         self.bin_count = list(bins)
         self.n_segments = nseg.value
-        self._ptrs.update(dict(zip(("row_order", "seg_row", "seg_begin", "hub_seg_ptr"), [p.value for p in sp])))
+        self._ptrs.update(dict(zip(("row_order", "seg_row", "seg_begin", "seg_end", "seg_slot", "hub_seg_ptr"),
+                                   [p.value for p in sp])))
 
     @property
     def handle(self):
@@ -217,6 +219,8 @@ class Csr:
     row_order = property(lambda self: self._view("row_order", self.n, torch.int32))
     seg_row = property(lambda self: self._view("seg_row", self.n_segments, torch.int32))
     seg_begin = property(lambda self: self._view("seg_begin", self.n_segments, torch.int32))
+    seg_end = property(lambda self: self._view("seg_end", self.n_segments, torch.int32))
+    seg_slot = property(lambda self: self._view("seg_slot", self.n_segments, torch.int32))
     hub_seg_ptr = property(lambda self: self._view("hub_seg_ptr", self.bin_count[4] + 1, torch.int32))
 
     def destroy(self):

@@ -23,6 +23,8 @@ struct GatherArgs {
     const int32_t* row_order;
     const int32_t* seg_row;
     const int32_t* seg_begin;
+    const int32_t* seg_end;
+    const int32_t* seg_slot;
     const void* x;
     void* out;
     float* partial;
@@ -114,12 +116,13 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     }
 
     const bool wide = WIDE && okq[VPL - 1];            // both vectors of the lane exist: one 32-byte load per entry
-    int32_t row = 0, b = 0, e = 0;
+    int32_t row = 0, b = 0, e = 0, part = 0;      // part: where a hub segment's partial sums go
     if (active) {
         if (rg.hub) {
             row = a.seg_row[slot];
             b = a.seg_begin[slot];
-            e = min(b + kHubSegment, a.row_ptr[row + 1]);
+            e = a.seg_end[slot];
+            part = a.seg_slot[slot];
         } else {
             row = a.row_order[rg.item_begin + slot];
             b = a.row_ptr[row];
@@ -244,7 +247,7 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         if (!okq[q]) continue;
         const int j = jq[q];
         if (rg.hub) {
-            float* p = a.partial + (int64_t)slot * a.fpad + j;
+            float* p = a.partial + (int64_t)part * a.fpad + j;
 #pragma unroll
             for (int i = 0; i < VECN; ++i)
                 if (j + i < chunk_end) p[i] = acc[q][i];
@@ -385,6 +388,7 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
     GatherArgs a;
     a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.edge_w = csr->edge_w; a.rdeg = csr->rdeg;
     a.row_order = csr->row_order; a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin;
+    a.seg_end = csr->seg_end; a.seg_slot = csr->seg_slot;
     a.x = d_x; a.out = d_out; a.partial = static_cast<float*>(d_scratch);
     a.ldx = ldx; a.ldo = ldo; a.f = f; a.chunk_width = cw;
     a.n_ctiles = (cw + lpr * vpl * elems - 1) / (lpr * vpl * elems);

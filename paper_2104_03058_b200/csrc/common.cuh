@@ -41,6 +41,8 @@ struct gnnfd_csr {
     const int32_t* row_order;
     const int32_t* seg_row;
     const int32_t* seg_begin;
+    const int32_t* seg_end;
+    const int32_t* seg_slot;
     const int32_t* hub_seg_ptr;
 };
 

@@ -489,37 +489,79 @@ finalize_entries(const u64* __restrict__ keys, const int32_t* __restrict__ vals,
     }
 }
 
-// segments per hub row; entry n_hub (one past the end) is 0 so that the scan yields the total
+// Hub rows are cut twice: at the boundaries of source ranges of `range_rows` vertex ids (a row's sources are
+// ascending, so a range is a contiguous piece of the row) and then into segments of at most GNNFD_HUB_SEGMENT
+// entries.  Segments are scheduled range by range (all hub rows' pieces of source range 0, then range 1, ...),
+// so the hub rows that are gathered at the same time read the same narrow band of x: a source that several
+// hub rows share is fetched from HBM once per sweep instead of once per row.  A segment keeps a second number,
+// its slot: slots count a row's segments in ascending source order, row after row, and index the partial
+// results, so that the per-row reductions run over a contiguous, ordered slot range.
+
+__device__ __forceinline__ int32_t lower_bound_col(const int32_t* __restrict__ col, int32_t lo, int32_t hi, int64_t bound)
+{
+    while (lo < hi) {
+        const int32_t mid = lo + ((hi - lo) >> 1);
+        if ((int64_t)col[mid] < bound) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// per hub row and source range: the number of segments (range-major: count[r * hub_cap + i]) and per hub row
+// the total; entries past the last hub row are 0 so that the scans yield the totals
 __global__ void __launch_bounds__(kThreads)
-hub_segment_counts(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ row_order, int64_t n,
-                   const BuildCounts* __restrict__ counts, int64_t hub_cap, int32_t* __restrict__ seg_count)
+hub_segment_counts(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                   const int32_t* __restrict__ row_order, int64_t n, const BuildCounts* __restrict__ counts, int64_t hub_cap,
+                   int32_t n_ranges, int64_t range_rows, int32_t* __restrict__ range_count, int32_t* __restrict__ seg_count)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (i > hub_cap) return;
     const int32_t n_hub = counts->bin_count[4];
-    int32_t c = 0;
+    int32_t total = 0;
     if (i < n_hub) {
         const int32_t v = row_order[n - n_hub + i];
-        c = (row_ptr[v + 1] - row_ptr[v] + kHubSegment - 1) / kHubSegment;
+        int32_t pos = row_ptr[v];
+        const int32_t e = row_ptr[v + 1];
+        for (int32_t r = 0; r < n_ranges; ++r) {
+            const int32_t nxt = r == n_ranges - 1 ? e : lower_bound_col(col_idx, pos, e, (int64_t)(r + 1) * range_rows);
+            const int32_t c = (nxt - pos + kHubSegment - 1) / kHubSegment;
+            range_count[(int64_t)r * hub_cap + i] = c;
+            total += c;
+            pos = nxt;
+        }
+    } else if (i < hub_cap) {
+        for (int32_t r = 0; r < n_ranges; ++r) range_count[(int64_t)r * hub_cap + i] = 0;
     }
-    seg_count[i] = c;
+    seg_count[i] = total;
+    if (i == 0) range_count[(int64_t)n_ranges * hub_cap] = 0;
 }
 
+// range_first: exclusive scan of range_count (the schedule position of a row's first segment in a range);
+// hub_seg_ptr: exclusive scan of seg_count (the row's first slot)
 __global__ void __launch_bounds__(kThreads)
-fill_segments(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ row_order, int64_t n,
-              BuildCounts* __restrict__ counts, const int32_t* __restrict__ hub_seg_ptr, int64_t hub_cap,
-              int32_t* __restrict__ seg_row, int32_t* __restrict__ seg_begin)
+fill_segments(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, const int32_t* __restrict__ row_order,
+              int64_t n, BuildCounts* __restrict__ counts, const int32_t* __restrict__ hub_seg_ptr,
+              const int32_t* __restrict__ range_first, int64_t hub_cap, int32_t n_ranges, int64_t range_rows,
+              int32_t* __restrict__ seg_row, int32_t* __restrict__ seg_begin, int32_t* __restrict__ seg_end,
+              int32_t* __restrict__ seg_slot)
 {
     const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     const int32_t n_hub = counts->bin_count[4];
     if (i == 0) counts->n_segments = hub_seg_ptr[n_hub];
     if (i >= hub_cap || i >= n_hub) return;
     const int32_t v = row_order[n - n_hub + i];
-    const int32_t b = row_ptr[v];
-    const int32_t first = hub_seg_ptr[i], last = hub_seg_ptr[i + 1];
-    for (int32_t s = first; s < last; ++s) {
-        seg_row[s] = v;
-        seg_begin[s] = b + (s - first) * kHubSegment;
+    int32_t pos = row_ptr[v];
+    const int32_t e = row_ptr[v + 1];
+    int32_t slot = hub_seg_ptr[i];
+    for (int32_t r = 0; r < n_ranges; ++r) {
+        const int32_t nxt = r == n_ranges - 1 ? e : lower_bound_col(col_idx, pos, e, (int64_t)(r + 1) * range_rows);
+        int32_t p = range_first[(int64_t)r * hub_cap + i];
+        for (int32_t x0 = pos; x0 < nxt; x0 += kHubSegment, ++p, ++slot) {
+            seg_row[p] = v;
+            seg_begin[p] = x0;
+            seg_end[p] = min(x0 + kHubSegment, nxt);
+            seg_slot[p] = slot;
+        }
+        pos = nxt;
     }
 }
 
@@ -533,6 +575,8 @@ struct BuildLayout {
     int64_t seg_cap;       // upper bound on hub segments
     int src_bits, key_bits, passes, digit_bits;
     int first_bit;         // lowest key bit the sort looks at (0; src_bits when rows keep their input order)
+    int n_ranges;          // source ranges the hub rows are cut at (1: no cut)
+    int64_t range_rows;    // vertex ids per source range
     int val_bits;          // > 0: keys and values share one 64-bit word (key << val_bits | value + 1)
 };
 
@@ -554,7 +598,12 @@ static int make_layout(int64_t n, int64_t e, uint32_t flags, BuildLayout* L)
     if (L->n_tiles == 0) L->n_tiles = 1;
     L->row_tiles = (n + kSortTile - 1) / kSortTile;
     L->hub_cap = m / (GNNFD_HUB_DEGREE + 1) + 1;
-    L->seg_cap = m / kHubSegment + L->hub_cap + 1;
+    // source ranges of 65,536 vertices (a 512-byte feature row each makes 32 MB, well inside L2), at most 64 of
+    // them; a row whose sources are not ascending (input-order build) cannot be cut by range
+    L->range_rows = GNNFD_HUB_RANGE_ROWS;
+    while ((n + L->range_rows - 1) / L->range_rows > 64) L->range_rows <<= 1;
+    L->n_ranges = (flags & GNNFD_CSR_INPUT_ORDER) ? 1 : (int)((n + L->range_rows - 1) / L->range_rows);
+    L->seg_cap = m / kHubSegment + L->hub_cap * L->n_ranges + 1;
     int bits = 1;
     while ((int64_t(1) << bits) < n) ++bits;
     int dst_bits = 1;
@@ -581,7 +630,7 @@ int64_t segment_capacity(int64_t n, int64_t e, uint32_t flags)
 }
 
 struct PersistentPtrs {
-    int32_t *row_ptr, *col_idx, *perm, *row_order, *seg_row, *seg_begin, *hub_seg_ptr;
+    int32_t *row_ptr, *col_idx, *perm, *row_order, *seg_row, *seg_begin, *seg_end, *seg_slot, *hub_seg_ptr;
     float *edge_w, *dinv, *rdeg;
     BuildCounts* counts;
 };
@@ -598,6 +647,8 @@ static void carve_persistent(Carver& c, int64_t n, const BuildLayout& L, Persist
     p->row_order = c.take<int32_t>((size_t)n);
     p->seg_row = c.take<int32_t>((size_t)L.seg_cap);
     p->seg_begin = c.take<int32_t>((size_t)L.seg_cap);
+    p->seg_end = c.take<int32_t>((size_t)L.seg_cap);
+    p->seg_slot = c.take<int32_t>((size_t)L.seg_cap);
     p->hub_seg_ptr = c.take<int32_t>((size_t)L.hub_cap + 1);
     p->counts = c.take<BuildCounts>(1);
 }
@@ -610,8 +661,8 @@ struct ScratchPtrs {
 static size_t flag_ints(int64_t n, const BuildLayout& L)
 {
     // one count per tile of the duplicate removal, a 64-bit dump for the row sort's keys (2 ints per row),
-    // hub segment counts
-    size_t a = (size_t)L.m / kUniqueTile + 2, b = 2 * (size_t)n + 2, c = (size_t)L.hub_cap + 1;
+    // hub segment counts (per source range and hub row, then per hub row)
+    size_t a = (size_t)L.m / kUniqueTile + 2, b = 2 * (size_t)n + 2, c = (size_t)L.hub_cap * (L.n_ranges + 1) + 4;
     size_t r = a > b ? a : b;
     return (r > c ? r : c) + 1;
 }
@@ -754,14 +805,18 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
         GNNFD_LAUNCH("radix_scatter", s, radix_scatter<true>, (unsigned)L.row_tiles, kScatterThreads, sizeof(ScatterSmem), keys_alt,
                      vals_alt, reinterpret_cast<u64*>(S.flags), P.row_order, n, 32, kRadix - 1, L.row_tiles, S.hist);
     }
-    // the flag buffer is free again: per-hub-row segment counts
-    int32_t* seg_count = S.flags;
+    // the flag buffer is free again: segment counts per (source range, hub row), then per hub row
+    int32_t* range_count = S.flags;
+    int32_t* seg_count = S.flags + (size_t)L.hub_cap * L.n_ranges + 1;
     GNNFD_LAUNCH("hub_segment_counts", s, hub_segment_counts, blocks_for((size_t)L.hub_cap + 1, kThreads), kThreads, 0,
-                 P.row_ptr, P.row_order, n, P.counts, L.hub_cap, seg_count);
+                 P.row_ptr, P.col_idx, P.row_order, n, P.counts, L.hub_cap, L.n_ranges, L.range_rows, range_count, seg_count);
     rc = exclusive_scan_i32(seg_count, P.hub_seg_ptr, (size_t)L.hub_cap + 1, S.scan_temp, s);
     if (rc) return rc;
-    GNNFD_LAUNCH("fill_segments", s, fill_segments, blocks_for((size_t)L.hub_cap, kThreads), kThreads, 0, P.row_ptr,
-                 P.row_order, n, P.counts, P.hub_seg_ptr, L.hub_cap, P.seg_row, P.seg_begin);
+    rc = exclusive_scan_i32(range_count, range_count, (size_t)L.hub_cap * L.n_ranges + 1, S.scan_temp, s);
+    if (rc) return rc;
+    GNNFD_LAUNCH("fill_segments", s, fill_segments, blocks_for((size_t)L.hub_cap, kThreads), kThreads, 0, P.row_ptr, P.col_idx,
+                 P.row_order, n, P.counts, P.hub_seg_ptr, range_count, L.hub_cap, L.n_ranges, L.range_rows, P.seg_row,
+                 P.seg_begin, P.seg_end, P.seg_slot);
     GNNFD_CUDA_CHECK(cudaGetLastError());
     GNNFD_CUDA_CHECK(cudaMemcpyAsync(&host_counts, P.counts, sizeof(BuildCounts), cudaMemcpyDeviceToHost, s));
     GNNFD_CUDA_CHECK(cudaStreamSynchronize(s));
@@ -789,6 +844,8 @@ int gnnfd_build_csr(int64_t n, int64_t e, const void* d_src, const void* d_dst, 
     h->row_order = P.row_order;
     h->seg_row = P.seg_row;
     h->seg_begin = P.seg_begin;
+    h->seg_end = P.seg_end;
+    h->seg_slot = P.seg_slot;
     h->hub_seg_ptr = P.hub_seg_ptr;
     *out = h;
     return GNNFD_OK;

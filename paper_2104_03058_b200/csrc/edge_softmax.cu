@@ -43,6 +43,8 @@ struct SoftmaxArgs {
     const int32_t* row_order;
     const int32_t* seg_row;
     const int32_t* seg_begin;
+    const int32_t* seg_end;
+    const int32_t* seg_slot;
     const int32_t* hub_seg_ptr;
     const float* s_src;
     const float* s_dst;
@@ -170,12 +172,13 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
     const int hb = sl % LPS;             // which block of HB heads of a slot
     const int sp = sl / LPS;             // which of the SP slots of a step
     const bool active = slot < rg.item_count;
-    int32_t row = 0, b = 0, e = 0;
+    int32_t row = 0, b = 0, e = 0, part = 0;      // part: where a hub segment's (max, sum) lives
     if (active) {
         if (rg.hub) {
             row = a.seg_row[slot];
             b = a.seg_begin[slot];
-            e = min(b + kHubSegment, a.row_ptr[row + 1]);
+            e = a.seg_end[slot];
+            part = a.seg_slot[slot];
         } else {
             row = a.row_order[rg.item_begin + slot];
             b = a.row_ptr[row];
@@ -234,7 +237,7 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
             if constexpr (MODE == kModeHubStats) {
                 if (active && head_ok && sp == 0) {
 #pragma unroll
-                    for (int h = 0; h < HB; ++h) a.seg_stats[(int64_t)slot * a.heads + h0 + h] = make_float2(m[h], l[h]);
+                    for (int h = 0; h < HB; ++h) a.seg_stats[(int64_t)part * a.heads + h0 + h] = make_float2(m[h], l[h]);
                 }
             }
 #pragma unroll
@@ -242,7 +245,7 @@ __device__ __forceinline__ void softmax_items(const SoftmaxArgs& a, const Range&
         } else {
 #pragma unroll
             for (int h = 0; h < HB; ++h) {
-                const float2 st = (active && head_ok) ? a.seg_stats[(int64_t)slot * a.heads + h0 + h] : make_float2(0.f, 0.f);
+                const float2 st = (active && head_ok) ? a.seg_stats[(int64_t)part * a.heads + h0 + h] : make_float2(0.f, 0.f);
                 m[h] = st.x;
                 inv[h] = st.y;
             }
@@ -391,7 +394,8 @@ int gnnfd_edge_softmax(const gnnfd_csr_t* csr, const float* d_s_src, const float
 
     SoftmaxArgs a;
     a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.row_order = csr->row_order;
-    a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin; a.hub_seg_ptr = csr->hub_seg_ptr;
+    a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin; a.seg_end = csr->seg_end; a.seg_slot = csr->seg_slot;
+    a.hub_seg_ptr = csr->hub_seg_ptr;
     a.s_src = d_s_src; a.s_dst = d_s_dst; a.alpha = d_alpha; a.seg_stats = static_cast<float2*>(d_scratch);
     a.slope = negative_slope; a.heads = heads; a.n_hub = (int32_t)csr->bin_count[4];
 

@@ -20,6 +20,8 @@ struct GatArgs {
     const int32_t* row_order;
     const int32_t* seg_row;
     const int32_t* seg_begin;
+    const int32_t* seg_end;
+    const int32_t* seg_slot;
     const float* s_src;
     const float* s_dst;
     const void* z;
@@ -115,12 +117,13 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         zq[q] = static_cast<const T*>(a.z) + (okq[q] ? j0 + q * VECN : col0);
     }
 
-    int32_t row = 0, b = 0, e = 0;
+    int32_t row = 0, b = 0, e = 0, part = 0;      // part: where a hub segment's partial results go
     if (active) {
         if (rg.hub) {
             row = a.seg_row[slot];
             b = a.seg_begin[slot];
-            e = min(b + kHubSegment, a.row_ptr[row + 1]);
+            e = a.seg_end[slot];
+            part = a.seg_slot[slot];
         } else {
             row = a.row_order[rg.item_begin + slot];
             b = a.row_ptr[row];
@@ -281,7 +284,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         // every lane of a head holds the same (m, l); the first lane of each head inside this column tile stores
         // it (sweeps that share a head store identical values)
         if (j0 % a.dim == 0 || c == 0) {
-            float* ml = a.partial_ml + ((int64_t)slot * a.heads + h) * 2;
+            float* ml = a.partial_ml + ((int64_t)part * a.heads + h) * 2;
             ml[0] = m;
             ml[1] = l;
         }
@@ -292,7 +295,7 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         if (!okq[q]) continue;
         const int j = j0 + q * VECN;
         if (rg.hub) {
-            float* p = a.partial + (int64_t)slot * a.fpad + j;
+            float* p = a.partial + (int64_t)part * a.fpad + j;
 #pragma unroll
             for (int i = 0; i < VECN; ++i)
                 if (j + i < chunk_end) p[i] = acc[q][i];
@@ -476,7 +479,7 @@ int gat_aggregate_impl(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnn
 
     GatArgs a;
     a.row_ptr = csr->row_ptr; a.col_idx = csr->col_idx; a.row_order = csr->row_order;
-    a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin;
+    a.seg_row = csr->seg_row; a.seg_begin = csr->seg_begin; a.seg_end = csr->seg_end; a.seg_slot = csr->seg_slot;
     a.s_src = g.s_src; a.s_dst = g.s_dst; a.z = d_z; a.out = d_out;
     a.partial = g.partial; a.partial_ml = g.partial_ml;
     a.ldz = ldz; a.ldo = ldo; a.slope = negative_slope;

@@ -246,7 +246,7 @@ int gnnfd_csr_info(const gnnfd_csr_t* csr, int64_t* n, int64_t* nnz, const int32
 
 int gnnfd_csr_schedule(const gnnfd_csr_t* csr, int64_t bin_count[5], const int32_t** d_row_order,
                        int64_t* n_segments, const int32_t** d_seg_row, const int32_t** d_seg_begin,
-                       const int32_t** d_hub_seg_ptr)
+                       const int32_t** d_seg_end, const int32_t** d_seg_slot, const int32_t** d_hub_seg_ptr)
 {
     if (!csr) return GNNFD_INVALID_ARG;
     if (bin_count)
@@ -255,6 +255,8 @@ int gnnfd_csr_schedule(const gnnfd_csr_t* csr, int64_t bin_count[5], const int32
     if (n_segments) *n_segments = csr->n_segments;
     if (d_seg_row) *d_seg_row = csr->seg_row;
     if (d_seg_begin) *d_seg_begin = csr->seg_begin;
+    if (d_seg_end) *d_seg_end = csr->seg_end;
+    if (d_seg_slot) *d_seg_slot = csr->seg_slot;
     if (d_hub_seg_ptr) *d_hub_seg_ptr = csr->hub_seg_ptr;
     return GNNFD_OK;
 }

@@ -95,12 +95,35 @@ def check_schedule(g, csr, deg):
     seg_ptr = csr.hub_seg_ptr.cpu().numpy()
     seg_row = csr.seg_row.cpu().numpy()
     seg_begin = csr.seg_begin.cpu().numpy()
+    seg_end = csr.seg_end.cpu().numpy()
+    seg_slot = csr.seg_slot.cpu().numpy()
     row_ptr = csr.row_ptr.cpu().numpy()
+    col = csr.col_idx.cpu().numpy()
     assert seg_ptr[0] == 0 and seg_ptr[-1] == csr.n_segments
+    assert sorted(seg_slot.tolist()) == list(range(csr.n_segments))          # every slot is scheduled exactly once
+    # source ranges: GNNFD_HUB_RANGE_ROWS ids, doubled until at most 64 cover the graph
+    width = g.HUB_RANGE_ROWS
+    while (n + width - 1) // width > 64:
+        width *= 2
+    by_slot = np.argsort(seg_slot)                                # schedule position of slot s
     for i, v in enumerate(hubs):
-        want = np.arange(row_ptr[v], row_ptr[v + 1], g.HUB_SEGMENT)
-        np.testing.assert_array_equal(seg_begin[seg_ptr[i]:seg_ptr[i + 1]], want)
-        assert (seg_row[seg_ptr[i]:seg_ptr[i + 1]] == v).all()
+        pos = by_slot[seg_ptr[i]:seg_ptr[i + 1]]                  # the row's segments in slot order
+        assert (seg_row[pos] == v).all()
+        b, e = seg_begin[pos], seg_end[pos]
+        # in slot order the segments tile the row: ascending, gap-free, none empty, none above the segment size
+        assert b[0] == row_ptr[v] and e[-1] == row_ptr[v + 1] and (b[1:] == e[:-1]).all()
+        assert ((e - b) > 0).all() and ((e - b) <= g.HUB_SEGMENT).all()
+        # a segment stays inside one source range, and a range's piece of the row is cut into as few segments as fit
+        r_first, r_last = col[b] // width, col[e - 1] // width
+        assert (r_first == r_last).all()
+        for r in np.unique(r_first):
+            piece = (e - b)[r_first == r]
+            assert len(piece) == (piece.sum() + g.HUB_SEGMENT - 1) // g.HUB_SEGMENT
+    # launch order: range by range, inside a range hub row by hub row (in row_order), inside a row ascending
+    if csr.n_segments:
+        hub_index = {int(v): i for i, v in enumerate(hubs)}
+        key = [(int(col[seg_begin[p]]) // width, hub_index[int(seg_row[p])], int(seg_begin[p])) for p in range(csr.n_segments)]
+        assert key == sorted(key)
 
 
 # ------------------------------------------------------------------ CSR build
@@ -309,6 +332,36 @@ def test_gat_general_shapes_with_hub_rows(g, heads, dim):
         got = g.aggregate_gat(csr, dev(z), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=width)
         assert_close_f32(got.cpu().numpy(), want, scale, "gat %dx%d width %d" % (heads, dim, width))
     s_src, s_dst = g.gat_scores(dev(z), dev(a_src), dev(a_dst), heads, dim)
+    alpha = g.edge_softmax(csr, s_src, s_dst, 0.2).cpu().numpy()
+    want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), 0.2)
+    assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
+
+
+def test_hub_rows_cut_at_source_ranges(g):
+    """More vertices than one source range holds: hub rows are cut at the range boundaries and their pieces are
+    launched range by range; partial results still combine per row in ascending source order."""
+    n = 3 * g.HUB_RANGE_ROWS + 1234                   # four source ranges, the last one nearly empty
+    src, dst = gg.uniform_graph(n, 400_000, seed=12)
+    rng = np.random.default_rng(12)
+    for i, (v, k) in enumerate(((5, 9000), (n - 1, 2500), (70_000, 3000))):
+        dst[i * 10_000:i * 10_000 + k] = v            # hub rows whose sources fall in every range
+    src[25_000:28_000] = rng.integers(0, 40_000, 3000)          # ... and one whose sources all lie in range 0
+    dst[25_000:28_000] = 99_999
+    csr, (row_ptr, col, _) = check_csr(g, n, src, dst, SL)
+    assert csr.bin_count[4] == 4 and csr.n_segments > 4 * 3
+    f, heads, dim = 16, 2, 8
+    x = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=12)
+    threads = orc.max_threads()
+    for model, fn in (("gcn", g.aggregate_gcn), ("sage", g.aggregate_sage)):
+        want, scale = orc.aggregate(model, row_ptr, col, x, f, threads=threads)
+        for width in (f, 4):
+            assert_close_f32(fn(csr, dev(x), f=f, chunk_width=width).cpu().numpy(), want, scale, model)
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=12, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=12, stream=6)
+    want, scale = orc.aggregate_gat(row_ptr, col, x, a_src, a_dst, heads, dim, 0.2, threads=threads)
+    got = g.aggregate_gat(csr, dev(x), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=8)
+    assert_close_f32(got.cpu().numpy(), want, scale, "gat")
+    s_src, s_dst = g.gat_scores(dev(x), dev(a_src), dev(a_dst), heads, dim)
     alpha = g.edge_softmax(csr, s_src, s_dst, 0.2).cpu().numpy()
     want_alpha = orc.edge_softmax(row_ptr, col, s_src.cpu().numpy(), s_dst.cpu().numpy(), 0.2)
     assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
