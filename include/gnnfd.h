@@ -82,7 +82,9 @@ typedef enum {
  */
 #define GNNFD_HUB_DEGREE 2048
 #define GNNFD_HUB_SEGMENT 1024
-#define GNNFD_HUB_RANGE_ROWS 65536
+#ifndef GNNFD_HUB_RANGE_ROWS
+#define GNNFD_HUB_RANGE_ROWS 524288
+#endif
 
 /* Sizes (bytes) of the two device buffers gnnfd_build_csr needs for n vertices and e input edges.
  * persistent: must stay alive and untouched while the handle is in use.

@@ -20,7 +20,7 @@ OK, INVALID_ARG, BAD_INDEX, TOO_LARGE, WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA_ER
 STATIC_SCRATCH_EXCEEDED = -7
 COMBINE_TF32, COMBINE_FP32 = 0, 1
 STATIC_SCRATCH_BYTES = 32 << 20
-HUB_DEGREE, HUB_SEGMENT, HUB_RANGE_ROWS = 2048, 1024, 65536
+HUB_DEGREE, HUB_SEGMENT, HUB_RANGE_ROWS = 2048, 1024, 524288
 
 _lib = None
 

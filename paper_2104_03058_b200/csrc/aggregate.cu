@@ -96,13 +96,12 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     constexpr int EPB = R * S;                            // entries per batch
     constexpr unsigned kFull = 0xffffffffu;
     const int tid = threadIdx.x;
-    const int slot = block_in_range * ROWS + tid / S;
+    const int group = tid / S;
     const int sl = tid % S;
     const int g = sl / LPR;
     const int c = sl % LPR;
     const int warp = tid >> 5, lane = tid & 31;
     const int seg = lane - sl;                   // first lane of this row's segment inside the warp
-    const bool active = slot < rg.item_count;
 
     int jq[VPL];
     bool okq[VPL];
@@ -114,8 +113,11 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
         okq[q] = jq[q] < chunk_end;
         xq[q] = static_cast<const T*>(a.x) + (okq[q] ? jq[q] : col0);   // out-of-chunk lanes re-read a valid column
     }
-
     const bool wide = WIDE && okq[VPL - 1];            // both vectors of the lane exist: one 32-byte load per entry
+    const uint32_t ld = (uint32_t)a.ldx;
+
+    const int slot = block_in_range * ROWS + group;
+    const bool active = slot < rg.item_count;
     int32_t row = 0, b = 0, e = 0, part = 0;      // part: where a hub segment's partial sums go
     if (active) {
         if (rg.hub) {
@@ -128,6 +130,15 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
             b = a.row_ptr[row];
             e = a.row_ptr[row + 1];
         }
+    }
+    int32_t ucur[R];
+    float wcur[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int32_t kk = b + r * S + sl;
+        const bool ok = kk < e;
+        ucur[r] = ok ? __ldcs(a.col_idx + kk) : -1;
+        wcur[r] = (WEIGHTED && ok) ? __ldcs(a.edge_w + kk) : 0.f;
     }
 
     // Two levels of accumulation: `acc` takes at most kChain products in a row, then moves into the
@@ -142,20 +153,9 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
         for (int i = 0; i < VECN; ++i) acc[q][i] = 0.f;
 
-    const uint32_t ld = (uint32_t)a.ldx;
     const int n_batches = __reduce_max_sync(kFull, (e - b + EPB - 1) / EPB);     // the warp loops together
     const bool two_level = n_batches > FLUSH;                                    // short rows never leave the first level
     if (two_level) second_level<VPL * VECN, true>(tot_s, tid, &acc[0][0], 0);
-
-    int32_t ucur[R];
-    float wcur[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int32_t kk = b + r * S + sl;
-        const bool ok = kk < e;
-        ucur[r] = ok ? __ldcs(a.col_idx + kk) : -1;
-        wcur[r] = (WEIGHTED && ok) ? __ldcs(a.edge_w + kk) : 0.f;
-    }
 
     for (int ib = 0; ib < n_batches; ++ib) {
         const int32_t kb = b + ib * EPB;
@@ -179,16 +179,28 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
             }
             __syncwarp();
         }
+        auto consume = [&](const Vec<T, VECN> (&v)[UB][VPL], const float (&wv)[UB]) {
 #pragma unroll
-        for (int s0 = 0; s0 < SPB; s0 += UB) {
-            Vec<T, VECN> v[UB][VPL];
-            float wv[UB];
-            if (full) {
+            for (int i = 0; i < UB; ++i)
+#pragma unroll
+                for (int q = 0; q < VPL; ++q)
+#pragma unroll
+                    for (int k = 0; k < VECN; ++k) {
+                        if (WEIGHTED) acc[q][k] = fmaf(wv[i], v[i][q].get(k), acc[q][k]);
+                        else acc[q][k] += v[i][q].get(k);
+                    }
+        };
+        if (full) {
+            // every lane has all of the batch's entries: straight-line code, no tests
+#pragma unroll
+            for (int s0 = 0; s0 < SPB; s0 += UB) {
+                Vec<T, VECN> v[UB][VPL];
+                float wv[UB];
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
-                    const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
-                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
+                    const int r = (s0 + i) / LPR, tt = (s0 + i) % LPR;
+                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + tt * EP + g] : ucur[r];
+                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + tt * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)u * ld;
                     if (WIDE && wide) {
                         load_pair(v[i][0], v[i][VPL - 1], xq[0] + off);
@@ -197,12 +209,23 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
                         for (int q = 0; q < VPL; ++q) v[i][q].load(xq[q] + off);
                     }
                 }
-            } else {
+                consume(v, wv);
+            }
+        } else {
+            // A ragged batch.  Step s works on entries s * EP .. of a row's batch, so the steps past the longest
+            // remainder in the warp have nothing to do for any lane (a row of 3 entries in a class whose batch
+            // holds 16 would otherwise pay for 16).
+            const int rem = __reduce_max_sync(kFull, e - kb);
+#pragma unroll
+            for (int s0 = 0; s0 < SPB; s0 += UB) {
+                if (s0 > 0 && s0 * EP >= rem) break;
+                Vec<T, VECN> v[UB][VPL];
+                float wv[UB];
 #pragma unroll
                 for (int i = 0; i < UB; ++i) {
-                    const int r = (s0 + i) / LPR, t = (s0 + i) % LPR;
-                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + t * EP + g] : ucur[r];
-                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + t * EP + g] : wcur[r];
+                    const int r = (s0 + i) / LPR, tt = (s0 + i) % LPR;
+                    const int32_t u = LPR > 1 ? stage_col[buf][warp][r * 32 + seg + tt * EP + g] : ucur[r];
+                    if (WEIGHTED) wv[i] = LPR > 1 ? stage_w[buf][warp][r * 32 + seg + tt * EP + g] : wcur[r];
                     const size_t off = (size_t)(uint32_t)max(u, 0) * ld;
                     if (WIDE && wide) {
                         if (u >= 0) load_pair(v[i][0], v[i][VPL - 1], xq[0] + off);
@@ -215,16 +238,8 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
                         }
                     }
                 }
+                consume(v, wv);
             }
-#pragma unroll
-            for (int i = 0; i < UB; ++i)
-#pragma unroll
-                for (int q = 0; q < VPL; ++q)
-#pragma unroll
-                    for (int k = 0; k < VECN; ++k) {
-                        if (WEIGHTED) acc[q][k] = fmaf(wv[i], v[i][q].get(k), acc[q][k]);
-                        else acc[q][k] += v[i][q].get(k);
-                    }
         }
 #pragma unroll
         for (int r = 0; r < R; ++r) { ucur[r] = unext[r]; wcur[r] = wnext[r]; }
@@ -240,29 +255,30 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
 #pragma unroll
             for (int i = 0; i < VECN; ++i) acc[q][i] += __shfl_down_sync(kFull, acc[q][i], o, S);
 
-    if (!active || g != 0) return;
-    const float scale = (WEIGHTED || rg.hub) ? 1.f : a.rdeg[row];
+    if (active && g == 0) {
+        const float scale = (WEIGHTED || rg.hub) ? 1.f : a.rdeg[row];
 #pragma unroll
-    for (int q = 0; q < VPL; ++q) {
-        if (!okq[q]) continue;
-        const int j = jq[q];
-        if (rg.hub) {
-            float* p = a.partial + (int64_t)part * a.fpad + j;
+        for (int q = 0; q < VPL; ++q) {
+            if (!okq[q]) continue;
+            const int j = jq[q];
+            if (rg.hub) {
+                float* p = a.partial + (int64_t)part * a.fpad + j;
 #pragma unroll
-            for (int i = 0; i < VECN; ++i)
-                if (j + i < chunk_end) p[i] = acc[q][i];
-            continue;
-        }
-        const int64_t o = (int64_t)row * a.ldo + j;
-        if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
+                for (int i = 0; i < VECN; ++i)
+                    if (j + i < chunk_end) p[i] = acc[q][i];
+                continue;
+            }
+            const int64_t o = (int64_t)row * a.ldo + j;
+            if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
 #pragma unroll
-            for (int i = 0; i < VECN; i += 4)
-                __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
-                       make_float4(acc[q][i] * scale, acc[q][i + 1] * scale, acc[q][i + 2] * scale, acc[q][i + 3] * scale));
-        } else {
+                for (int i = 0; i < VECN; i += 4)
+                    __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
+                           make_float4(acc[q][i] * scale, acc[q][i + 1] * scale, acc[q][i + 2] * scale, acc[q][i + 3] * scale));
+            } else {
 #pragma unroll
-            for (int i = 0; i < VECN; ++i)
-                if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[q][i] * scale);
+                for (int i = 0; i < VECN; ++i)
+                    if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[q][i] * scale);
+            }
         }
     }
 }
