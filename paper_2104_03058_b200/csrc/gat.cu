@@ -117,13 +117,12 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         zq[q] = static_cast<const T*>(a.z) + (okq[q] ? j0 + q * VECN : col0);
     }
 
-    int32_t row = 0, b = 0, e = 0, part = 0;      // part: where a hub segment's partial results go
+    int32_t row = 0, b = 0, e = 0;
     if (active) {
         if (rg.hub) {
             row = a.seg_row[slot];
             b = a.seg_begin[slot];
             e = a.seg_end[slot];
-            part = a.seg_slot[slot];
         } else {
             row = a.row_order[rg.item_begin + slot];
             b = a.row_ptr[row];
@@ -194,12 +193,8 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         // one group of UB entries: gathers issued together, then one update of the running softmax
         auto steps = [&](auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
-            // in a ragged batch step s works on entries s * EP .. of a row's batch: the steps past the longest
-            // remainder in the warp have nothing to do for any lane
-            const int rem = FULL ? EPB : __reduce_max_sync(kFull, e - kb);
 #pragma unroll
             for (int s0 = 0; s0 < SPB; s0 += UB) {
-                if (!FULL && s0 > 0 && s0 * EP >= rem) break;
                 Vec<T, VECN> v[UB][VPL];
                 float lg[UB];
                 bool valid[UB];
@@ -284,6 +279,8 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
     }
 
     if (!active || g != 0 || !lane_ok) return;
+    // where a hub segment's partial results go (read here, at the end, so that it occupies no register during the walk)
+    const int32_t part = rg.hub ? a.seg_slot[slot] : 0;
     if (rg.hub) {
         // every lane of a head holds the same (m, l); the first lane of each head inside this column tile stores
         // it (sweeps that share a head store identical values)
