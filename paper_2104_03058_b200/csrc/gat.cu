@@ -31,6 +31,7 @@ struct GatArgs {
     int64_t ldz, ldo;
     float slope;
     int32_t f, heads, dim, chunk_width, n_ctiles, blocks_per_tile, fpad, out_bf16, wide_ok;
+    int32_t chunk_base;      // first chunk of this launch (a launch covers at most 65,535 chunks)
     int32_t n_ranges;
     Range range[kMaxRanges];
 };
@@ -310,15 +311,20 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
 }
 
 template <typename T, int VECN, int LPR, int VPL>
-__global__ void __launch_bounds__(kBlock) gat_aggregate(const __grid_constant__ GatArgs a)
+// Register budget: left to itself the compiler gives the wide instantiations anything between 80 and 126
+// registers from one build to the next (two blocks per SM instead of three, 20 % slower); three blocks per SM for
+// the vector-pair forms and four for the others is what the measured-good builds had.
+__global__ void __launch_bounds__(kBlock, (VPL == 2 && VECN > 1) ? 3 : 4) gat_aggregate(const __grid_constant__ GatArgs a)
 {
     __shared__ int32_t stage_col[2][kBlock / 32][kStageSlots];
     __shared__ float tot_s[VPL * VECN + 1][kBlock];        // second-level sums and denominator, one column per thread
-    const int64_t per_chunk = (int64_t)a.blocks_per_tile * a.n_ctiles;
-    const int chunk = (int)(blockIdx.x / per_chunk);
-    const int rem = (int)(blockIdx.x % per_chunk);
-    const int rb = rem / a.n_ctiles;
-    const int ctile = rem % a.n_ctiles;
+    // grid: x = (block of the sweep, column tile), y = chunk; blocks are issued x first, so the sweeps follow each
+    // other chunk by chunk.  (The chunk used to be divided out of a linear 64-bit block number: two 64-bit
+    // divisions per thread, more instructions than a short row's whole walk.)
+    const int chunk = a.chunk_base + (int)blockIdx.y;
+    const unsigned n_ct = (unsigned)a.n_ctiles;
+    const int rb = n_ct == 1 ? (int)blockIdx.x : (int)(blockIdx.x / n_ct);
+    const int ctile = n_ct == 1 ? 0 : (int)(blockIdx.x % n_ct);
     const int chunk_begin = chunk * a.chunk_width;
     const int chunk_end = min(a.f, chunk_begin + a.chunk_width);
     const int col0 = chunk_begin + ctile * (LPR * VPL * VECN);
@@ -494,13 +500,17 @@ int gat_aggregate_impl(const gnnfd_csr_t* csr, const void* d_z, int64_t ldz, gnn
 
     const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges);
     a.blocks_per_tile = (int32_t)blocks;
-    const int64_t grid = blocks * a.n_ctiles * n_chunks;
-    if (grid > 0x7fffffffll || blocks > 0x7fffffffll) return GNNFD_TOO_LARGE;
-    if (grid > 0) {
+    const int64_t grid_x = blocks * a.n_ctiles;
+    if (grid_x > 0x7fffffffll) return GNNFD_TOO_LARGE;
+    if (grid_x > 0) {
         GatKernel kernel;
         if (zdt == GNNFD_F32) kernel = vec ? pick_vpl<float, 4>(lpr, vpl) : pick_vpl<float, 1>(lpr, vpl);
         else kernel = vec ? pick_vpl<__nv_bfloat16, 8>(lpr, vpl) : pick_vpl<__nv_bfloat16, 1>(lpr, vpl);
-        GNNFD_LAUNCH("gat_aggregate", s, kernel, (unsigned)grid, kBlock, 0, a);
+        for (int c0 = 0; c0 < n_chunks; c0 += kMaxGridY) {
+            a.chunk_base = c0;
+            const dim3 grid((unsigned)grid_x, (unsigned)(n_chunks - c0 < kMaxGridY ? n_chunks - c0 : kMaxGridY));
+            GNNFD_LAUNCH("gat_aggregate", s, kernel, grid, kBlock, 0, a);
+        }
     }
     const int64_t n_hub = csr->bin_count[4];
     if (n_hub > 0) {
