@@ -284,90 +284,6 @@ __device__ __forceinline__ void gather_rows(const GatherArgs& a, const Range& rg
     }
 }
 
-// Rows of up to 32 entries (the two lowest degree classes): LPR lanes own a row and walk its entries four at a
-// time, every lane reading the row's indices and weights itself (one broadcast transaction per group).  The
-// batched walk above costs a short row as many instructions as a full batch of entries; here a row of three
-// entries costs three entries' worth plus a short prologue, which is what these classes are bound by.
-template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, bool WIDE>
-__device__ __forceinline__ void gather_short_rows(const GatherArgs& a, const Range& rg, int block_in_range, int col0, int chunk_end)
-{
-    constexpr int ROWS = kBlock / LPR;
-    constexpr int U = 4;                               // entries in flight
-    const int tid = threadIdx.x;
-    const int slot = block_in_range * ROWS + tid / LPR;
-    const int c = tid % LPR;
-    if (slot >= rg.item_count) return;
-    int jq[VPL];
-    bool okq[VPL];
-    const T* xq[VPL];
-#pragma unroll
-    for (int q = 0; q < VPL; ++q) {
-        jq[q] = col0 + (WIDE ? c * VPL + q : c + q * LPR) * VECN;
-        okq[q] = jq[q] < chunk_end;
-        xq[q] = static_cast<const T*>(a.x) + (okq[q] ? jq[q] : col0);   // out-of-chunk lanes re-read a valid column
-    }
-    const bool wide = WIDE && okq[VPL - 1];
-    const uint32_t ld = (uint32_t)a.ldx;
-    const int32_t row = a.row_order[rg.item_begin + slot];
-    const int32_t b = a.row_ptr[row], e = a.row_ptr[row + 1];
-    float acc[VPL][VECN];
-#pragma unroll
-    for (int q = 0; q < VPL; ++q)
-#pragma unroll
-        for (int i = 0; i < VECN; ++i) acc[q][i] = 0.f;
-    for (int32_t k = b; k < e; k += U) {
-        int32_t u[U];
-        float w[U];
-#pragma unroll
-        for (int i = 0; i < U; ++i) {
-            const bool ok = k + i < e;
-            u[i] = ok ? __ldg(a.col_idx + k + i) : -1;
-            w[i] = (WEIGHTED && ok) ? __ldg(a.edge_w + k + i) : 0.f;
-        }
-        Vec<T, VECN> v[U][VPL];
-#pragma unroll
-        for (int i = 0; i < U; ++i) {
-            const size_t off = (size_t)(uint32_t)max(u[i], 0) * ld;
-            if (WIDE && wide) {
-                if (u[i] >= 0) load_pair(v[i][0], v[i][VPL - 1], xq[0] + off);
-                else { v[i][0].zero(); v[i][VPL - 1].zero(); }
-            } else {
-#pragma unroll
-                for (int q = 0; q < VPL; ++q) {
-                    if (u[i] >= 0) v[i][q].load(xq[q] + off);
-                    else v[i][q].zero();
-                }
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < U; ++i)
-#pragma unroll
-            for (int q = 0; q < VPL; ++q)
-#pragma unroll
-                for (int kk = 0; kk < VECN; ++kk) {
-                    if (WEIGHTED) acc[q][kk] = fmaf(w[i], v[i][q].get(kk), acc[q][kk]);
-                    else acc[q][kk] += v[i][q].get(kk);
-                }
-    }
-    const float scale = WEIGHTED ? 1.f : a.rdeg[row];
-#pragma unroll
-    for (int q = 0; q < VPL; ++q) {
-        if (!okq[q]) continue;
-        const int j = jq[q];
-        const int64_t o = (int64_t)row * a.ldo + j;
-        if (VECN % 4 == 0 && a.out_vec_ok && j + VECN <= chunk_end) {
-#pragma unroll
-            for (int i = 0; i < VECN; i += 4)
-                __stcs(reinterpret_cast<float4*>(static_cast<float*>(a.out) + o + i),
-                       make_float4(acc[q][i] * scale, acc[q][i + 1] * scale, acc[q][i + 2] * scale, acc[q][i + 3] * scale));
-        } else {
-#pragma unroll
-            for (int i = 0; i < VECN; ++i)
-                if (j + i < chunk_end) store_elem(a.out, a.out_bf16, o + i, acc[q][i] * scale);
-        }
-    }
-}
-
 template <typename T, int VECN, int LPR, int VPL, bool WEIGHTED, bool WIDE = false>
 __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggregate(const __grid_constant__ GatherArgs a)
 {
@@ -391,10 +307,6 @@ __global__ void __launch_bounds__(kBlock, GNNFD_GATHER_MIN_BLOCKS) gather_aggreg
         if (i < a.n_ranges && rb >= a.range[i].first_block) r = i;
     const Range rg = a.range[r];
     const int bir = rb - rg.first_block;
-    if (rg.short_rows) {
-        gather_short_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE>(a, rg, bir, col0, chunk_end);
-        return;
-    }
     switch (rg.ep_log2) {
         case 0: gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 1>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
         case 1: if constexpr (LPR * 2 <= 32) gather_rows<T, VECN, LPR, VPL, WEIGHTED, WIDE, 2>(a, rg, bir, col0, chunk_end, stage_col, stage_w, tot_s); break;
@@ -510,7 +422,7 @@ static int aggregate(bool weighted, const gnnfd_csr_t* csr, const void* d_x, int
                 (n_chunks == 1 || (cw * xsize) % 32 == 0);
     a.out_vec_ok = odt == GNNFD_F32 && ((uintptr_t)d_out % 16 == 0) && (ldo % 4 == 0) && (n_chunks == 1 || cw % 4 == 0);
 
-    const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges, true);
+    const int64_t blocks = plan_ranges(csr, lpr, a.range, &a.n_ranges);
     a.blocks_per_tile = (int32_t)blocks;
     const int64_t grid_x = blocks * a.n_ctiles;
     if (grid_x > 0x7fffffffll) return GNNFD_TOO_LARGE;

@@ -19,7 +19,6 @@ struct Range {
     int32_t item_count;
     int32_t ep_log2;       // log2 of the edge-parallel groups per row
     int32_t hub;           // 1: items are hub segments writing partial results
-    int32_t short_rows;    // 1: rows of up to 32 entries, for a kernel that has a leaner walk for them
 };
 
 inline int ilog2(int x) { int l = 0; while ((1 << l) < x) ++l; return l; }
@@ -45,24 +44,22 @@ inline int ep_for_bin(int bin, int lpr)
     return want[bin] < cap ? want[bin] : cap;
 }
 
-// Fills ranges for `lpr` lanes per row; returns the blocks of one column tile of one sweep.  `short_walk`: the
-// kernel walks rows of the two lowest degree classes with `lpr` lanes each, whatever ep_for_bin says.
-inline int64_t plan_ranges(const gnnfd_csr_t* csr, int lpr, Range* range, int32_t* n_ranges, bool short_walk = false)
+// Fills ranges for `lpr` lanes per row; returns the blocks of one column tile of one sweep.
+inline int64_t plan_ranges(const gnnfd_csr_t* csr, int lpr, Range* range, int32_t* n_ranges)
 {
     int nr = 0;
     int64_t blocks = 0;
     if (csr->n_segments > 0) {
         const int ep = ep_for_bin(4, lpr);
         const int rows_per_block = kBlock / (lpr * ep);
-        range[nr++] = Range{(int32_t)blocks, 0, (int32_t)csr->n_segments, ilog2(ep), 1, 0};
+        range[nr++] = Range{(int32_t)blocks, 0, (int32_t)csr->n_segments, ilog2(ep), 1};
         blocks += (csr->n_segments + rows_per_block - 1) / rows_per_block;
     }
     for (int bin = 3; bin >= 0; --bin) {
         if (csr->bin_count[bin] == 0) continue;
-        const int short_rows = (short_walk && bin <= 1) ? 1 : 0;
-        const int ep = short_rows ? 1 : ep_for_bin(bin, lpr);
+        const int ep = ep_for_bin(bin, lpr);
         const int rows_per_block = kBlock / (lpr * ep);
-        range[nr++] = Range{(int32_t)blocks, (int32_t)csr->bin_start[bin], (int32_t)csr->bin_count[bin], ilog2(ep), 0, short_rows};
+        range[nr++] = Range{(int32_t)blocks, (int32_t)csr->bin_start[bin], (int32_t)csr->bin_count[bin], ilog2(ep), 0};
         blocks += (csr->bin_count[bin] + rows_per_block - 1) / rows_per_block;
     }
     *n_ranges = nr;
