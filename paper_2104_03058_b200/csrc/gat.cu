@@ -194,8 +194,12 @@ __device__ __forceinline__ void gat_rows(const GatArgs& a, const Range& rg, int 
         // one group of UB entries: gathers issued together, then one update of the running softmax
         auto steps = [&](auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
+            // in a ragged batch step s works on entries s * EP .. of a row's batch: the steps past the longest
+            // remainder in the warp have nothing to do for any lane
+            const int rem = FULL ? EPB : __reduce_max_sync(kFull, e - kb);
 #pragma unroll
             for (int s0 = 0; s0 < SPB; s0 += UB) {
+                if (!FULL && s0 > 0 && s0 * EP >= rem) break;
                 Vec<T, VECN> v[UB][VPL];
                 float lg[UB];
                 bool valid[UB];
