@@ -63,8 +63,8 @@ WORKLOADS["reddit_small_gat_hid64"] = (
     "GAT on the config-4 recipe at 1/4 of the vertices and 1/16 of the edges, 8 heads x 8 dims fp32")
 # DRAM bytes per launch of the dominant kernel from a one-pass ncu capture of the same launch
 # (dram__bytes_read.sum + dram__bytes_write.sum), valid only for the kernel sources they were taken with.
-NCU_TRAFFIC = {"config4": {"bytes": 16.830e9, "sources_sha1": "12924cfb3529b0f63b04404dbb56de9979e7f414"},
-               "config5_f256": {"bytes": 18.517e9, "sources_sha1": "12924cfb3529b0f63b04404dbb56de9979e7f414"}}
+NCU_TRAFFIC = {"config4": {"bytes": 16.823e9, "sources_sha1": "20fda6161c29e4d7927491bed812043bb79b7a77"},
+               "config5_f256": {"bytes": 14.644e9, "sources_sha1": "20fda6161c29e4d7927491bed812043bb79b7a77"}}
 KERNEL_SOURCES = ("paper_2104_03058_b200/csrc/aggregate.cu", "paper_2104_03058_b200/csrc/schedule.cuh",
                   "paper_2104_03058_b200/csrc/vec.cuh")
 # L2-to-crossbar peak that ncu derives on this part (derived__lts__lts2xbar_bytes.sum.peak_sustained), bytes per clock
@@ -467,7 +467,7 @@ def run_ours(args):
 
     combine_ms = combine_fp32_ms = None
     layer_ms = {}
-    if not bf16 and args.combine_out > 0 and not by_columns:
+    if not bf16 and args.combine_out > 0 and not by_columns and not args.core_only:
         # the dense transform a layer runs ahead of its aggregation (Section III), timed alone: x [n, f] -> [n, combine_out];
         # then whole layers (transform + aggregation of the transformed columns) on the built CSR
         co = args.combine_out
@@ -496,7 +496,7 @@ def run_ours(args):
     # the light set-up for graphs that are aggregated once: destination-only sort (rows in edge-id order), then
     # the same aggregation; and both in one call from one buffer
     light = None
-    if not gat and not by_columns and not (w.flags & g.CSR_DEDUP):
+    if not gat and not by_columns and not (w.flags & g.CSR_DEDUP) and not args.core_only:
         def light_step():
             c2 = g.build_csr(w.n, d_src, d_dst, w.flags | g.CSR_INPUT_ORDER, persistent=persistent, scratch=scratch)
             (g.aggregate_sage if w.model == "sage" else g.aggregate_gcn)(c2, d_x, f=w.f, chunk_width=cw, out=out_view,
@@ -658,6 +658,8 @@ def main():
                     help="destination rows in the CPU-oracle sample (0: 16384 per step of --impl reference, "
                          "98304 for the one cpu_baseline step of the CUDA arm)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--core-only", action="store_true",
+                    help="leave out the side measurements (dense transform, layers, one-shot path): for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
