@@ -85,3 +85,28 @@ def test_more_ranks_than_chunks_leaves_idle_ranks_without_work():
     before = g.launch_count()
     assert sharding.aggregate_slab(csr, x, "gcn", f, 16, 4, 3, out) == (16, 16)      # one chunk, rank 3 of 4: nothing to do
     assert g.launch_count() == before
+
+
+def test_slab_gather_over_nccl_with_device_tensors():
+    """gather_slabs_ on CUDA tensors through the NCCL backend.  One GPU is what a test gets, so the group has one
+    rank: the collective runs on the device and must leave the rank's own columns and the padding as they are."""
+    import os
+    import socket
+
+    import torch.distributed as dist
+    from paper_2104_03058_b200 import sharding
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        out = torch.arange(300 * 20, dtype=torch.float32, device="cuda").reshape(300, 20).contiguous()
+        want = out.clone()
+        sharding.gather_slabs_(out, 17, 4)
+        torch.cuda.synchronize()
+        assert torch.equal(out, want)
+        ms, units = sharding.reduce_job_timing(3.5, 10.0, device=torch.device("cuda", 0))
+        assert (ms, units) == (3.5, 10.0)
+    finally:
+        dist.destroy_process_group()

@@ -168,3 +168,41 @@ def test_config5_full_size_csr_and_bf16_aggregation():
     for width in (64, 8):
         got = g.aggregate_gcn(csr, xd, f=w.f, chunk_width=width)[sel].cpu().numpy()
         assert (np.abs(got - want) <= 1e-2 * np.abs(want) + 1e-5 * scale + 1e-6).all(), "width %d" % width
+
+
+def test_config5_full_size_input_width_256():
+    """Config 5 at the input width (F = 256 bf16, 1.07 GB of features, the launch `bench.py --workload config5_f256`
+    times): sampled rows of every degree class (hub rows are cut at four source ranges on this graph) against the
+    oracle, undecomposed and at chunk width 64; a sentinel shows that every output element is written; two runs
+    give the same bits."""
+    import paper_2104_03058_b200 as g
+    w = gg.config5(f=256)
+    row_ptr, col, _ = orc.build_csr(w.n, w.src, w.dst, w.flags)
+    csr = g.build_csr(w.n, torch.from_numpy(w.src).cuda(), torch.from_numpy(w.dst).cuda(), w.flags)
+    assert csr.nnz == len(col) and csr.bin_count[4] > 0
+    # the hub rows' segments span several source ranges
+    seg_first = csr.col_idx[csr.seg_begin.long()].cpu().numpy() // g.HUB_RANGE_ROWS
+    assert len(np.unique(seg_first)) == (w.n + g.HUB_RANGE_ROWS - 1) // g.HUB_RANGE_ROWS == 4
+    deg = np.diff(row_ptr)
+    rng = np.random.default_rng(9)
+    by_class = [np.flatnonzero((deg > lo) & (deg <= hi)) for lo, hi in ((0, 8), (8, 32), (32, 128), (128, 2048), (2048, 1 << 30))]
+    rows = np.unique(np.concatenate([rng.choice(c, min(len(c), 48), replace=False) for c in by_class] +
+                                    [np.argsort(deg)[-4:]])).astype(np.int64)
+    want, scale = orc.aggregate("gcn", row_ptr, col, w.x, w.f, rows=rows, threads=orc.max_threads())
+    xd = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16)
+    sel = torch.from_numpy(rows).cuda()
+    out = torch.full((w.n, w.f), float("nan"), device="cuda")
+    first = None
+    for width in (256, 64, 256):
+        out.fill_(float("nan"))
+        g.aggregate_gcn(csr, xd, f=w.f, chunk_width=width, out=out)
+        assert not bool(torch.isnan(out).any()), "width %d left elements unwritten" % width
+        got = out[sel].cpu().numpy()
+        assert (np.abs(got - want) <= 1e-2 * np.abs(want) + 1e-5 * scale + 1e-6).all(), "width %d" % width
+        # the fp32 bar alone holds too: bf16 inputs are widened exactly, only the summation order differs
+        assert (np.abs(got - want) <= 1e-5 * scale + 1e-6).all(), "width %d (fp32 bar)" % width
+        if width == 256:
+            if first is None:
+                first = out.clone()
+            else:
+                assert torch.equal(out, first)
