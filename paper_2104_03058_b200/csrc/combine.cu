@@ -47,13 +47,14 @@ constexpr uint64_t kWaitNs = 1000000000ull; // one second on one barrier before 
 constexpr int kSmemBudget = 100 * 1024;     // per block, so that two blocks share an SM
 constexpr int kSmemBudgetSplit = 108 * 1024; // fp32-faithful mode (hi and lo tiles per stage): still two blocks per SM
 constexpr int kSmemBudgetMax = 200 * 1024;  // fp32-faithful mode with wide tiles: one block per SM
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 6;
 
 struct CombineArgs {
     void* z;
     int64_t ldz;
     int32_t n, f_in, f_out, tile_n, stages, tmem_cols, z_bf16;
     int32_t acc_cols, n_main;   // tensor-memory columns per accumulator; accumulators the K blocks rotate over
+    int32_t xlo_col;            // first tensor-memory column of the x_lo ring (32 columns per stage), XT kernels only
     int32_t* status;        // set to 1 when a wait ran out (may be null)
     // GAT scores formed in the epilogue (all null / 0 when not wanted): a_src / a_dst [heads * dim] over the
     // output columns, s_src / s_dst [n, heads]
@@ -172,6 +173,35 @@ __device__ __forceinline__ void mma(uint32_t tmem_d, uint64_t desc_a, uint64_t d
     }
 }
 
+// tf32 MMA whose A operand (128 rows x 8 K elements, one 32-bit column per element, row = lane) lies in tensor memory
+__device__ __forceinline__ void mma_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t"
+        "}"
+        :
+        : "r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// 32 consecutive columns of the calling thread's lane (a warp covers 32 lanes)
+__device__ __forceinline__ void tmem_store_32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        :
+        : "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
 // arrives on the barrier once every MMA issued so far by this thread has finished
 __device__ __forceinline__ void mma_commit(uint64_t* bar)
 {
@@ -215,11 +245,15 @@ __device__ __forceinline__ void score_step(ScoreState& st, float val, int col, c
 
 // SPLIT: fp32-faithful mode (fp32 operands as tf32 hi + lo pairs, three MMAs per K slice); launched with
 // kSplitThreads threads, of which warps 2.. compute the lo tiles.
-template <bool BF16, bool SPLIT>
+// XT (with SPLIT): the lo part of the x tile is kept in tensor memory and fed to the MMA as its A operand from
+// there (warps 4 - 7 own one row each: they read it out of the swizzled stage, subtract the tf32 cut and store 32
+// columns), so a stage holds only x, w and w_lo in shared memory and the ring is a stage deeper.
+template <bool BF16, bool SPLIT, bool XT = false>
 __global__ void __launch_bounds__(SPLIT ? kSplitThreads : kCombineThreads)
 combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CombineArgs a)
 {
     static_assert(!(BF16 && SPLIT), "bf16 operands are used as they are");
+    static_assert(!XT || SPLIT, "x_lo in tensor memory belongs to the fp32-faithful mode");
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], split_bar[kMaxStages], accum_bar;
     __shared__ uint32_t tmem_base_slot;
@@ -229,11 +263,12 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
     // the dynamic buffer is aligned to 1024 bytes by hand (the swizzle pattern repeats every 1024 bytes)
     unsigned char* tiles = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int kTileK = kTileKBytes / (BF16 ? 2 : 4);      // elements of K per stage
-    constexpr int kSplitWarps = SPLIT ? kSplitThreads / 32 - 2 : 0;
+    constexpr int kSplitWarps = !SPLIT ? 0 : XT ? 4 : kSplitThreads / 32 - 2;
     const uint32_t a_bytes = kTileM * kTileKBytes;
     const uint32_t b_bytes = (uint32_t)a.tile_n * kTileKBytes;
     const uint32_t stage_bytes = a_bytes + b_bytes;            // what the TMA unit delivers per stage
-    const uint32_t stage_pitch = SPLIT ? 2 * stage_bytes : stage_bytes;   // the lo tiles follow the loaded ones
+    // the lo tiles follow the loaded ones (with XT only w's: x_lo lives in tensor memory)
+    const uint32_t stage_pitch = !SPLIT ? stage_bytes : XT ? stage_bytes + b_bytes : 2 * stage_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row0 = blockIdx.x * kTileM;
@@ -308,10 +343,16 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
                     // the two small products go to an accumulator of their own (the last one), where they lose nothing
                     // against the large sum; the epilogue adds it once
                     const uint32_t acc_lo = tmem_base + (uint32_t)(a.n_main * a.acc_cols);
-                    const uint64_t da_lo = operand_desc(a_addr + stage_bytes + k * kMmaKBytes);
-                    const uint64_t db_lo = operand_desc(b_addr + stage_bytes + k * kMmaKBytes);
-                    mma<BF16>(acc_lo, da_lo, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    mma<BF16>(acc_lo, da, db_lo, idesc, 1u);
+                    if constexpr (XT) {
+                        const uint64_t db_lo = operand_desc(a_addr + stage_bytes + k * kMmaKBytes);
+                        mma_a_tmem(acc_lo, tmem_base + (uint32_t)(a.xlo_col + s * 32 + k * 8), db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        mma<BF16>(acc_lo, da, db_lo, idesc, 1u);
+                    } else {
+                        const uint64_t da_lo = operand_desc(a_addr + stage_bytes + k * kMmaKBytes);
+                        const uint64_t db_lo = operand_desc(b_addr + stage_bytes + k * kMmaKBytes);
+                        mma<BF16>(acc_lo, da_lo, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        mma<BF16>(acc_lo, da, db_lo, idesc, 1u);
+                    }
                     mma<BF16>(acc, da, db, idesc, carry);
                 } else {
                     mma<BF16>(acc, da, db, idesc, carry);
@@ -321,7 +362,7 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
         }
         if (ok) mma_commit(&accum_bar);
         else *(volatile int*)&abort_flag = 1;
-    } else if (SPLIT && warp >= 2) {
+    } else if (SPLIT && !XT && warp >= 2) {
         // lo tiles: element by element over the stage (the swizzle only permutes 16-byte pieces, so the lo tile
         // has the layout of the loaded one), then visible to the tensor core's reads, then one arrival per warp
         const int t = threadIdx.x - 64;
@@ -345,6 +386,46 @@ combine_mma(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ C
                 lo[i] = r;
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&split_bar[s]);
+        }
+        if (!ok && lane == 0) *(volatile int*)&abort_flag = 1;
+    } else if (SPLIT && XT && warp >= 4) {
+        // x_lo into tensor memory: thread t of warps 4 - 7 owns row t of the tile (lane t of tensor memory).  The
+        // stage stores row r's 16-byte piece c at position c ^ (r & 7) (128-byte swizzle); w_lo as above.
+        const int t = threadIdx.x - 128;
+        const int n_vec_w = (int)(b_bytes / 16);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % a.stages;
+            ok = mbar_wait(&full_bar[s], (kb / a.stages) & 1, a.wait_ns);
+            ok = __all_sync(0xffffffffu, ok && !*(volatile int*)&abort_flag);
+            if (!ok) break;
+            const unsigned char* stage = tiles + (size_t)s * stage_pitch;
+            uint32_t lo_bits[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 v = *reinterpret_cast<const float4*>(stage + (size_t)t * kTileKBytes + ((c ^ (t & 7)) << 4));
+                lo_bits[4 * c + 0] = __float_as_uint(v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u));
+                lo_bits[4 * c + 1] = __float_as_uint(v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u));
+                lo_bits[4 * c + 2] = __float_as_uint(v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u));
+                lo_bits[4 * c + 3] = __float_as_uint(v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u));
+            }
+            tmem_store_32(tmem_base + ((uint32_t)((warp - 4) * 32) << 16) + (uint32_t)(a.xlo_col + s * 32), lo_bits);
+            const float4* hi = reinterpret_cast<const float4*>(stage + a_bytes);
+            float4* lo = reinterpret_cast<float4*>(const_cast<unsigned char*>(stage) + stage_bytes);
+            for (int i = t; i < n_vec_w; i += 128) {
+                const float4 v = hi[i];
+                float4 r;
+                r.x = v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+                r.y = v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+                r.z = v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+                r.w = v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+                lo[i] = r;
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&split_bar[s]);
         }
@@ -520,22 +601,50 @@ int combine_impl(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int
     if (scores && n_col_tiles > 1 && a.tile_n % dim != 0) return GNNFD_UNSUPPORTED;
     a.acc_cols = 32;
     while (a.acc_cols < a.tile_n) a.acc_cols <<= 1;
-    const int stage_bytes = (kTileM + a.tile_n) * kTileKBytes * (split ? 2 : 1);
-    int budget = split ? kSmemBudgetSplit : kSmemBudget;
-    bool two_per_sm = true;
-    if (budget / stage_bytes < 2) { budget = kSmemBudgetMax; two_per_sm = false; }      // wide tiles: one block per SM
-    // tensor memory: 512 columns per SM, shared by the blocks resident there; all of a block's share becomes accumulators
-    a.tmem_cols = two_per_sm ? 256 : 512;
-    const int n_acc = a.tmem_cols / a.acc_cols;
-    a.n_main = split ? n_acc - 1 : n_acc;
-    if (a.n_main < 1) return GNNFD_UNSUPPORTED;
-    a.stages = budget / stage_bytes;
-    if (a.stages > kMaxStages) a.stages = kMaxStages;
-    if (a.stages < 2) return GNNFD_UNSUPPORTED;
-    size_t smem = (size_t)a.stages * stage_bytes + 1024;
-    // each block takes half of the SM's tensor memory, so no more than two may share an SM (a third would sit in
-    // its allocation until one of them left): ask for more than a third of the SM's shared memory
-    if (smem < 80 * 1024) smem = 80 * 1024;
+    // Shared memory per stage, blocks per SM, tensor memory.  Tensor memory has 512 columns per SM, shared by the
+    // blocks resident there; a block takes its whole share: accumulators first and, in the fp32-faithful mode when
+    // it fits, a ring of 32 columns per stage for the lo part of the x tile (`xt`).
+    bool xt = false;
+    int stage_bytes = 0;
+    size_t smem = 0;
+    a.xlo_col = 0;
+    if (split) {
+        const int stage_xt = (kTileM + 2 * a.tile_n) * kTileKBytes;          // x, w, w_lo
+        for (int pass = 0; pass < 2 && !xt; ++pass) {
+            const int budget = pass == 0 ? kSmemBudgetSplit : kSmemBudgetMax;
+            const int tmem = pass == 0 ? 256 : 512;
+            int stages = budget / stage_xt;
+            if (stages > kMaxStages) stages = kMaxStages;
+            const int n_acc = stages >= 2 ? (tmem - stages * 32) / a.acc_cols : 0;
+            if (n_acc >= 2) {
+                xt = true;
+                stage_bytes = stage_xt;
+                a.stages = stages;
+                a.tmem_cols = tmem;
+                a.n_main = n_acc - 1;
+                a.xlo_col = tmem - stages * 32;
+            }
+        }
+    }
+    if (!xt) {
+        stage_bytes = (kTileM + a.tile_n) * kTileKBytes * (split ? 2 : 1);
+        int budget = split ? kSmemBudgetSplit : kSmemBudget;
+        bool two_per_sm = true;
+        if (budget / stage_bytes < 2) { budget = kSmemBudgetMax; two_per_sm = false; }      // wide tiles: one block per SM
+        a.tmem_cols = two_per_sm ? 256 : 512;
+        const int n_acc = a.tmem_cols / a.acc_cols;
+        a.n_main = split ? n_acc - 1 : n_acc;
+        if (a.n_main < 1) return GNNFD_UNSUPPORTED;
+        a.stages = budget / stage_bytes;
+        if (a.stages > kMaxStages) a.stages = kMaxStages;
+        if (a.stages < 2) return GNNFD_UNSUPPORTED;
+    }
+    smem = (size_t)a.stages * stage_bytes + 1024;
+    // a block that takes half of the SM's tensor memory must not meet a third one on its SM (it would sit in its
+    // allocation until one of the others left); one that takes all of it must be alone: size the shared-memory
+    // request accordingly
+    if (a.tmem_cols == 256 && smem < 80 * 1024) smem = 80 * 1024;
+    if (a.tmem_cols == 512 && smem < 120 * 1024) smem = 120 * 1024;
 
     CUtensorMap map_x, map_w;
     if (!make_map(&map_x, d_x, bf16, n, f_in, ldx, kTileM) || !make_map(&map_w, d_w_t, bf16, f_out, f_in, ldw, a.tile_n)) {
@@ -546,6 +655,9 @@ int combine_impl(int64_t n, const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, int
     if (bf16) {
         GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         GNNFD_LAUNCH("combine_bf16", s, (combine_mma<true, false>), grid, kCombineThreads, smem, map_x, map_w, a);
+    } else if (split && xt) {
+        GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GNNFD_LAUNCH("combine_fp32_3xtf32", s, (combine_mma<false, true, true>), grid, kSplitThreads, smem, map_x, map_w, a);
     } else if (split) {
         GNNFD_CUDA_CHECK(cudaFuncSetAttribute(combine_mma<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         GNNFD_LAUNCH("combine_fp32_3xtf32", s, (combine_mma<false, true>), grid, kSplitThreads, smem, map_x, map_w, a);
