@@ -533,6 +533,27 @@ def test_gat_many_and_odd_head_counts(g, heads, dim):
     assert (np.abs(alpha - want_alpha) <= 1e-5 * want_alpha + 1e-7).all()
 
 
+def test_more_chunks_than_one_launch_covers(g):
+    """70,000 decomposition layers of one column each: a launch covers at most 65,535 chunks (grid y), so the
+    aggregation goes out as two launches; every column must still come back right."""
+    n, f = 40, 70_000
+    src, dst = gg.uniform_graph(n, 200, seed=8)
+    x = gg.features_f32(n, f, dist="normal", p0=0, p1=1, seed=8)
+    row_ptr, col, _ = orc.build_csr(n, src, dst, SL)
+    csr = g.build_csr(n, dev(src), dev(dst), SL)
+    before = g.launch_count()
+    want, scale = orc.aggregate("gcn", row_ptr, col, x, f)
+    got = g.aggregate_gcn(csr, dev(x), f=f, chunk_width=1)
+    assert g.launch_count() - before == 2
+    assert_close_f32(got.cpu().numpy(), want, scale, "gcn, 70,000 chunks")
+    heads, dim = f // 8, 8
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=8, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0, p1=0.3, seed=8, stream=6)
+    want, scale = orc.aggregate_gat(row_ptr, col, x, a_src, a_dst, heads, dim, 0.2)
+    got = g.aggregate_gat(csr, dev(x), dev(a_src), dev(a_dst), heads, dim, 0.2, chunk_width=1)
+    assert_close_f32(got.cpu().numpy(), want, scale, "gat, 70,000 chunks")
+
+
 def test_int64_ids_beyond_int32_are_rejected(g):
     src = torch.tensor([0, 2 ** 31 + 5], dtype=torch.int64, device="cuda")
     dst = torch.tensor([1, 2], dtype=torch.int64, device="cuda")
