@@ -223,6 +223,15 @@ int gnnfd_oneshot_sage(int64_t n, int64_t e, const void* d_src, const void* d_ds
                        const void* d_x, int64_t ldx, gnnfd_dtype_t xdt, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
                        int32_t f, int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
 
+/* The same for the attention aggregator (defined in the GAT section below; arguments as for gnnfd_aggregate_gat). */
+int gnnfd_oneshot_gat_workspace_bytes(int64_t n, int64_t e, uint32_t flags, int32_t heads, int32_t dim,
+                                      size_t* scratch_bytes);
+
+int gnnfd_oneshot_gat(int64_t n, int64_t e, const void* d_src, const void* d_dst, gnnfd_itype_t itype, uint32_t flags,
+                      const void* d_z, int64_t ldz, gnnfd_dtype_t zdt, const float* d_a_src, const float* d_a_dst,
+                      int32_t heads, int32_t dim, float negative_slope, void* d_out, int64_t ldo, gnnfd_dtype_t odt,
+                      int32_t chunk_width, void* d_scratch, size_t scratch_bytes, void* stream);
+
 /* ------------------------------------------------------------------ GAT
  *
  * The attention aggregator is the third model the paper evaluates (Section II-A lists it with GCN and

@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
         one = [i64, i64, vp, vp, i32, u32, vp, i64, i32, vp, i64, i32, i32, i32, vp, sz, vp]
         L.gnnfd_oneshot_gcn.argtypes = one
         L.gnnfd_oneshot_sage.argtypes = one
+        L.gnnfd_oneshot_gat_workspace_bytes.argtypes = [i64, i64, u32, i32, i32, pp(sz)]
+        L.gnnfd_oneshot_gat.argtypes = [i64, i64, vp, vp, i32, u32, vp, i64, i32, vp, vp, i32, i32, fl, vp, i64, i32, i32,
+                                        vp, sz, vp]
         L.gnnfd_default_chunk_candidates.argtypes = [i32, i32, pp(i32), ctypes.c_int]
         L.gnnfd_tune_chunk_width.argtypes = [vp, ctypes.c_int, vp, i64, i32, vp, i64, i32, i32, pp(i32), ctypes.c_int,
                                              vp, sz, vp, pp(i32), pp(fl)]
@@ -334,6 +337,41 @@ def oneshot(model: str, n: int, src: torch.Tensor, dst: torch.Tensor, x: torch.T
               I32 if src.dtype == torch.int32 else I64, flags, xp, ldx, _dtype_code(x), op, ldo, _dtype_code(out), f,
               chunk_width, ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
               _stream_ptr(stream)), "gnnfd_oneshot_" + model)
+    return out
+
+
+def oneshot_gat(n: int, src: torch.Tensor, dst: torch.Tensor, z: torch.Tensor, a_src: torch.Tensor, a_dst: torch.Tensor,
+                heads: int, dim: int, negative_slope: float = 0.2, flags: int = 0, chunk_width: int | None = None,
+                out: torch.Tensor | None = None, out_dtype=None, scratch=None, stream=None):
+    """gnnfd_oneshot_gat: light build + GAT aggregation of a COO edge list in one call."""
+    if not (src.is_cuda and dst.is_cuda) or src.dtype != dst.dtype or src.shape != dst.shape or src.dim() != 1:
+        raise ValueError("src and dst must be 1-D CUDA tensors of the same dtype and length")
+    if src.dtype not in (torch.int32, torch.int64):
+        raise TypeError("edge ids must be int32 or int64")
+    src, dst = src.contiguous(), dst.contiguous()
+    f = heads * dim
+    chunk_width = f if chunk_width is None else chunk_width
+    if out is None:
+        out = torch.empty((n, f), dtype=out_dtype or torch.float32, device=z.device)
+    zp, ldz = _matrix(z, f, "z")
+    op, ldo = _matrix(out, f, "out")
+    _same_device(src.device, dst=dst, z=z, out=out)
+    _need_rows(z, n, "z")
+    _need_rows(out, n, "out")
+    _no_overlap(z, out, "z", "out")
+    a_src, a_dst = _attention_vectors(a_src, a_dst, heads, dim, z.device, stream)
+    if scratch is None:
+        need = ctypes.c_size_t()
+        _check(lib().gnnfd_oneshot_gat_workspace_bytes(n, src.numel(), flags, heads, dim, ctypes.byref(need)),
+               "gnnfd_oneshot_gat_workspace_bytes")
+        scratch = _alloc_bytes(need.value, z.device, stream)
+    _same_device(src.device, scratch=scratch)
+    _check(lib().gnnfd_oneshot_gat(n, src.numel(), ctypes.c_void_p(src.data_ptr()), ctypes.c_void_p(dst.data_ptr()),
+                                   I32 if src.dtype == torch.int32 else I64, flags, zp, ldz, _dtype_code(z),
+                                   ctypes.c_void_p(a_src.data_ptr()), ctypes.c_void_p(a_dst.data_ptr()), heads, dim,
+                                   negative_slope, op, ldo, _dtype_code(out), chunk_width,
+                                   ctypes.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
+                                   _stream_ptr(stream)), "gnnfd_oneshot_gat")
     return out
 
 

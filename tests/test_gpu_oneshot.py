@@ -96,6 +96,22 @@ def test_oneshot_matches_the_oracle_and_is_repeatable(model, flags):
     assert close(g.oneshot(model, w.n, src, dst, xb, flags=flags).cpu().numpy(), want16, scale16)
 
 
+@pytest.mark.parametrize("flags", [SL, SY | DD | SL])
+def test_oneshot_gat_matches_the_oracle(flags):
+    import paper_2104_03058_b200 as g
+    w = gg.scaled("config4", 0.05)                       # hub rows included
+    heads, dim = 4, 8
+    z = np.ascontiguousarray(w.x[:, :heads * dim])
+    a_src = gg.features_f32(heads, dim, dist="normal", p0=0.0, p1=0.3, seed=2, stream=5)
+    a_dst = gg.features_f32(heads, dim, dist="normal", p0=0.0, p1=0.3, seed=2, stream=6)
+    row_ptr, col, _ = orc.build_csr(w.n, w.src, w.dst, flags)
+    want, scale = orc.aggregate_gat(row_ptr, col, z, a_src, a_dst, heads, dim, 0.2)
+    for width in (heads * dim, dim):
+        got = g.oneshot_gat(w.n, dev(w.src), dev(w.dst), dev(z), dev(a_src), dev(a_dst), heads, dim, 0.2, flags=flags,
+                            chunk_width=width)
+        assert close(got.cpu().numpy(), want, scale), (flags, width)
+
+
 def test_oneshot_reports_bad_ids_and_small_buffers():
     import paper_2104_03058_b200 as g
     n, f = 50, 8
